@@ -1,0 +1,355 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle.
+
+Each test names the passage or the fact it rests on.  None of them needs a GPU.
+"""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import litevar_oracle as orc
+from paper_2411_17178_b200 import workloads as wlmod
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+S256 = wlmod.SCALES_256
+S512 = wlmod.SCALES_512
+S2K = wlmod.SCALES_2K
+
+
+# ---------------------------------------------------------------- schedule (Section 2)
+def test_worked_example_k2_shape():
+    # Section 2: "when k=2, the attention map has a shape of [4,5]"
+    assert orc.map_shape(S256, 2) == (4, 5)
+
+
+def test_256px_cumulative_tokens():
+    # Section 2, implementation details: the ten scales (1,2,3,4,5,6,8,10,13,16)
+    assert orc.offsets(S256)[1:] == [1, 5, 14, 30, 55, 91, 155, 255, 424, 680]
+    assert orc.map_shape(S256, 10) == (256, 680)
+    assert orc.map_shape(S512, 10) == (1024, 2240)
+    assert orc.map_shape(S2K, 14) == (16384, 34240)
+    assert sum(n * L for n, L in (orc.map_shape(S256, k) for k in range(1, 11))) == 286_434
+
+
+def test_parts_k_minus_2_first_part_14_columns():
+    # Section 2 step (2): k-2 parts, the first holds sum_{i<=3} s_i^2 = 14 columns
+    for k in range(4, 11):
+        p = orc.parts(S256, k)
+        assert len(p) == k - 2
+        assert p[0] == (0, 14)
+        assert p[-1][1] == orc.map_shape(S256, k)[1]
+        for (a0, a1), (b0, b1) in zip(p[:-1], p[1:]):
+            assert a1 == b0
+        # every later part is one scale: width s_j^2
+        assert [c1 - c0 for c0, c1 in p[1:]] == [s * s for s in S256[3:k]]
+    for k in (1, 2, 3):
+        assert len(orc.parts(S256, k)) == 1
+
+
+# ---------------------------------------------------------------- mask geometry
+def _live_rational(scales, k, w_row, q, t):
+    """Third formulation, exact rationals: locate the key cell that contains the query
+    cell's centre by interval membership, then Chebyshev distance in key cells."""
+    s_k = scales[k - 1]
+    off = [0]
+    for s in scales:
+        off.append(off[-1] + s * s)
+    j = next(j for j in range(1, k + 1) if off[j - 1] <= t < off[j])
+    s_j = scales[j - 1]
+    w = w_row[j - 1]
+    if w < 0:
+        return True
+    r, c = q // s_k, q % s_k
+    tt = t - off[j - 1]
+    rk, ck = tt // s_j, tt % s_j
+
+    def cell(x):
+        ctr = (Fraction(x) + Fraction(1, 2)) / s_k
+        hits = [i for i in range(s_j) if Fraction(i, s_j) <= ctr < Fraction(i + 1, s_j)]
+        assert len(hits) == 1
+        return hits[0]
+
+    return max(abs(rk - cell(r)), abs(ck - cell(c))) <= w
+
+
+@pytest.mark.parametrize("scales", [(1, 2, 3, 4), (1, 2, 3, 4, 5), (1, 2, 3, 4, 6, 9), (2, 3, 5, 7, 4)])
+@pytest.mark.parametrize("rho", [(1, 8), (1, 4), (1, 2)])
+def test_mask_brute_force_rationals(scales, rho):
+    w = orc.window_table(scales, rho=rho, n_global_scales=3)
+    for k in range(1, len(scales) + 1):
+        n_k, L_k = orc.map_shape(scales, k)
+        m = orc.mask(scales, k, w[k - 1])
+        assert m.shape == (n_k, L_k)
+        for q in range(n_k):
+            for t in range(L_k):
+                ref = _live_rational(scales, k, list(w[k - 1]), q, t)
+                assert orc.live(scales, k, w[k - 1], q, t) == ref
+                assert bool(m[q, t]) == ref
+
+
+def test_hand_count_1234_w1():
+    # scales (1,2,3,4), k=4, radius 1 on scale 4: 16 queries x 14 global keys, plus the
+    # own-scale part: per axis the clipped windows hold 2,3,3,2 cells -> (2+3+3+2)^2.
+    w = [-1, -1, -1, 1]
+    assert orc.live_count((1, 2, 3, 4), 4, w) == 16 * 14 + (2 + 3 + 3 + 2) ** 2 == 324
+
+
+def _closed_form_count(scales, k, w_row):
+    """Separable mask: a part's live entries = A^2, A = sum over query rows of the clipped
+    1-D window length (computed here with min/max clipping, not with |.| <= w)."""
+    s_k = scales[k - 1]
+    total = 0
+    for j in range(1, k + 1):
+        s_j = scales[j - 1]
+        w = w_row[j - 1]
+        if w < 0:
+            total += s_k * s_k * s_j * s_j
+            continue
+        A = 0
+        for x in range(s_k):
+            c = math.floor((x + 0.5) * s_j / s_k + 1e-12)
+            A += min(s_j - 1, c + w) - max(0, c - w) + 1
+        total += A * A
+    return total
+
+
+@pytest.mark.parametrize("scales,rho", [(S256, (1, 4)), (S512, (1, 4)), (S256, (1, 8)), (S256, (1, 2))])
+def test_live_counts_closed_form(scales, rho):
+    w = orc.window_table(scales, rho=rho)
+    for k in range(1, len(scales) + 1):
+        assert orc.live_count(scales, k, w[k - 1]) == _closed_form_count(scales, k, list(w[k - 1]))
+
+
+def test_live_counts_golden_file():
+    # values written by tests/golden/make_golden.py (calls only the oracle); the closed
+    # form above checks the same numbers independently.
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "live_counts.txt")) if l.strip() and l[0] != "#"]
+    assert rows
+    for name, rn, rd, k, dense, kept in rows:
+        scales = {"256": S256, "512": S512, "2k": S2K}[name]
+        w = orc.window_table(scales, rho=(int(rn), int(rd)))
+        k = int(k)
+        n_k, L_k = orc.map_shape(scales, k)
+        assert n_k * L_k == int(dense)
+        assert _closed_form_count(scales, k, list(w[k - 1])) == int(kept)
+
+
+def test_2k_final_step_counts_closed_form():
+    for rho in ((1, 8), (1, 4), (1, 2)):
+        w = orc.window_table(S2K, rho=rho)
+        cf = _closed_form_count(S2K, 14, list(w[13]))
+        # enumerate a strided subset of query rows with the oracle and compare per row
+        rows = list(range(0, 16384, 97))
+        m = orc.mask(S2K, 14, w[13], q_rows=rows)
+        s_k = 128
+        for i, q in enumerate(rows):
+            r, c = divmod(q, s_k)
+            per = 0
+            for j in range(1, 15):
+                s_j = S2K[j - 1]
+                wj = int(w[13, j - 1])
+                if wj < 0:
+                    per += s_j * s_j
+                    continue
+                lr = min(s_j - 1, orc.centre(r, s_j, s_k) + wj) - max(0, orc.centre(r, s_j, s_k) - wj) + 1
+                lc = min(s_j - 1, orc.centre(c, s_j, s_k) + wj) - max(0, orc.centre(c, s_j, s_k) - wj) + 1
+                per += lr * lc
+            assert int(m[i].sum()) == per
+        assert 0 < cf < 16384 * 34240
+
+
+def test_mask_invariants():
+    for scales in (S256, S512):
+        K = len(scales)
+        tables = [orc.window_table(scales, rho=r) for r in ((1, 8), (1, 4), (1, 2), (1, 1))]
+        for k in range(1, K + 1):
+            ms = [orc.mask(scales, k, t[k - 1]) for t in tables]
+            # nested in the radius
+            for a, b in zip(ms[:-1], ms[1:]):
+                assert not (a & ~b).any()
+            off = orc.offsets(scales)
+            m = ms[1]
+            # scales 1..3 fully live (attention-sink parts kept global)
+            assert m[:, :off[min(k, 3)]].all()
+            # the own-scale part is symmetric and contains the diagonal (co-located key)
+            own = m[:, off[k - 1]:off[k]]
+            assert (own == own.T).all()
+            assert own.diagonal().all()
+            # every query keeps at least one key in every part (radius >= 0)
+            for j in range(1, k + 1):
+                assert m[:, off[j - 1]:off[j]].any(axis=1).all()
+
+
+def test_r0_equal_1_is_full_attention_mask():
+    # Section 2: R_0 = 1 falls back to full attention
+    for k in range(1, 11):
+        assert orc.mask(S256, k, orc.full_table(S256)[k - 1]).all()
+    # a radius that covers the grid gives the same mask
+    big = orc.window_table(S256, rho=(4, 1))
+    assert orc.mask(S256, 10, big[9]).all()
+
+
+def test_literal_three_parts_variant():
+    # alternative reading of "first three parts": scales 1..5 global -> 55 global columns at 256px
+    w = orc.window_table(S256, n_global_scales=5)
+    m = orc.mask(S256, 10, w[9])
+    assert m[:, :55].all() and not m[:, 55:].all()
+
+
+# ---------------------------------------------------------------- savings (Table 1, abstract)
+def test_default_window_saving_close_to_table1():
+    # Table 1, threshold 0.95: 70.34 % FLOPs saving.  The synthetic default (rho = 1/4,
+    # three global scales) is a stand-in chosen to land within one point of it.
+    s = orc.schedule_saving(S256, orc.window_table(S256))
+    assert abs(100 * s - 70.34) < 1.0
+    assert abs(100 * s - 69.46) < 0.01
+    assert orc.schedule_saving(S256, orc.full_table(S256)) == 0.0     # Table 1, threshold 1 -> 0.00
+
+
+def test_asc_halves_what_mdwa_leaves():
+    # abstract: 85.2 % reduction with MDWA + ASC = 1 - (1 - 0.7034)/2
+    assert abs(100 * orc.flops_saving_with_asc(0.7034) - 85.2) < 0.05
+
+
+# ---------------------------------------------------------------- attention numerics
+def _rand(shape, seed):
+    return wlmod.randn_bf16(shape, seed)
+
+
+def test_full_window_equals_library_softmax_attention():
+    # R_0 = 1: plain softmax attention over the L_k prefix; checked against torch's SDPA in fp64.
+    scales = (1, 2, 3, 4, 5, 6)
+    k = 6
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((2, 3, n_k, 64), 1), _rand((2, 3, L_k + 7, 64), 2), _rand((2, 3, L_k + 7, 64), 3)
+    out = orc.attention_step(scales, k, orc.full_table(scales)[k - 1], Q, Kc, Vc)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        Q.double(), Kc[:, :, :L_k].double(), Vc[:, :, :L_k].double()).numpy()
+    assert np.abs(out - ref).max() < 1e-12
+
+
+def test_windowed_equals_library_attention_with_bool_mask():
+    scales = (1, 2, 3, 4, 5, 6, 8)
+    k = 7
+    w = orc.window_table(scales)
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((2, 2, n_k, 64), 4), _rand((2, 2, L_k, 64), 5), _rand((2, 2, L_k, 64), 6)
+    out = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc, sm_scale=0.2)
+    # mask built here pair by pair with the rational formulation, not with the oracle's
+    m = torch.tensor([[_live_rational(scales, k, list(w[k - 1]), q, t) for t in range(L_k)]
+                      for q in range(n_k)])
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        Q.double(), Kc.double(), Vc.double(), attn_mask=m, scale=0.2).numpy()
+    assert np.abs(out - ref).max() < 1e-12
+
+
+def test_attention_pure_python_loops_tiny():
+    # definition written out with scalar loops on a tiny case (catches transposed operands,
+    # a dropped scale, a wrong normaliser)
+    scales = (1, 2, 3, 4)
+    k = 4
+    w = [-1, -1, 0, 1]
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((2, 1, n_k, 64), 7), _rand((2, 1, L_k, 64), 8), _rand((2, 1, L_k, 64), 9)
+    out, wts = orc.attention_step(scales, k, w, Q, Kc, Vc, return_weights=True)
+    Qd, Kd, Vd = Q.double().numpy(), Kc.double().numpy(), Vc.double().numpy()
+    for b in range(2):
+        for q in range(n_k):
+            z = []
+            for t in range(L_k):
+                if _live_rational(scales, k, w, q, t):
+                    z.append((t, sum(Qd[b, 0, q, i] * Kd[b, 0, t, i] for i in range(64)) / 8.0))
+            mx = max(v for _, v in z)
+            den = sum(math.exp(v - mx) for _, v in z)
+            o = [0.0] * 64
+            for t, v in z:
+                p = math.exp(v - mx) / den
+                assert abs(wts[b, 0, q, t] - p) < 1e-13
+                for i in range(64):
+                    o[i] += p * Vd[b, 0, t, i]
+            assert np.abs(out[b, 0, q] - np.array(o)).max() < 1e-12
+
+
+def test_weights_rows_sum_to_one_and_masked_are_zero():
+    scales = S256[:8]
+    k = 8
+    w = orc.window_table(scales)
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((2, 2, n_k, 64), 10), _rand((2, 2, L_k, 64), 11), _rand((2, 2, L_k, 64), 12)
+    out, wts = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc, return_weights=True)
+    assert np.abs(wts.sum(-1) - 1.0).max() < 1e-12
+    m = orc.mask(scales, k, w[k - 1])
+    assert (wts[:, :, ~m] == 0.0).all()
+    assert (wts[:, :, m] > 0.0).all()
+
+
+def test_zero_queries_give_mean_of_live_values():
+    # closed form: q = 0 -> uniform weights over live keys -> out = mean of the live V rows
+    scales = (1, 2, 3, 4, 5)
+    k = 5
+    w = orc.window_table(scales)
+    n_k, L_k = orc.map_shape(scales, k)
+    Q = torch.zeros(2, 1, n_k, 64, dtype=torch.bfloat16)
+    Kc, Vc = _rand((2, 1, L_k, 64), 13), _rand((2, 1, L_k, 64), 14)
+    out = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc)
+    Vd = Vc.double().numpy()
+    for q in range(n_k):
+        idx = [t for t in range(L_k) if _live_rational(scales, k, list(w[k - 1]), q, t)]
+        assert np.abs(out[0, 0, q] - Vd[0, 0, idx].mean(0)).max() < 1e-12
+
+
+def test_dominant_key_selects_its_value_and_dead_key_is_ignored():
+    scales = (1, 2, 3, 4, 5)
+    k = 5
+    w = orc.window_table(scales)
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((2, 1, n_k, 64), 15), _rand((2, 1, L_k, 64), 16), _rand((2, 1, L_k, 64), 17)
+    q = 0
+    m = orc.mask(scales, k, w[k - 1])
+    dead = int(np.where(~m[q])[0][0])
+    livek = int(np.where(m[q])[0][-1])
+    base = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc)
+    # a dead key with a huge score must not change row q
+    K2 = Kc.clone()
+    K2[:, :, dead] = Q[:, :, q] * 50
+    V2 = Vc.clone()
+    V2[:, :, dead] = 1000.0
+    out2 = orc.attention_step(scales, k, w[k - 1], Q, K2, V2)
+    assert np.array_equal(out2[:, :, q], base[:, :, q])
+    # a live key with a huge score takes all the weight
+    K3 = Kc.clone()
+    K3[:, :, livek] = Q[:, :, q] * 50
+    out3 = orc.attention_step(scales, k, w[k - 1], Q, K3, Vc)
+    assert np.abs(out3[:, :, q] - Vc[:, :, livek].double().numpy()).max() < 1e-9
+
+
+def test_asc_copies_conditional_rows_and_ignores_unconditional_inputs():
+    scales = (1, 2, 3, 4, 5)
+    k = 5
+    w = orc.window_table(scales)
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((4, 2, n_k, 64), 18), _rand((4, 2, L_k, 64), 19), _rand((4, 2, L_k, 64), 20)
+    out = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc, share_cfg=True)
+    assert np.array_equal(out[2:], out[:2])
+    plain = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc)
+    assert np.array_equal(out[:2], plain[:2])
+    Q2 = Q.clone()
+    Q2[2:] = 7.0
+    out2 = orc.attention_step(scales, k, w[k - 1], Q2, Kc, Vc, share_cfg=True)
+    assert np.array_equal(out2, out)
+
+
+def test_sampled_rows_match_full_evaluation():
+    scales = S256[:7]
+    k = 7
+    w = orc.window_table(scales)
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((2, 2, n_k, 64), 21), _rand((2, 2, L_k, 64), 22), _rand((2, 2, L_k, 64), 23)
+    full = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc, share_cfg=True)
+    samples = [(0, 0, 0), (1, 1, 63), (0, 1, 17), (1, 0, 40)]
+    got = orc.attention_sampled(scales, k, w[k - 1], Q, Kc, Vc, samples, share_cfg=True)
+    for i, (b, h, q) in enumerate(samples):
+        assert np.abs(got[i] - full[b, h, q]).max() < 1e-13
