@@ -1,0 +1,178 @@
+/*
+ * litevar.h -- C ABI of the LiteVAR attention library for NVIDIA B200 (sm_100a).
+ *
+ * One operation: the attention that a VAR image generator runs at every coarse-to-fine
+ * scale step (the current scale's queries against the K/V cache of all scales so far),
+ * under LiteVAR's multi-diagonal window mask (MDWA, paper Section 2) and with LiteVAR's
+ * attention sharing across classifier-free guidance (ASC, paper Section 3).
+ *
+ * Notation (paper Section 2).  Scales s_1..s_K; scale k holds n_k = s_k^2 tokens in
+ * row-major order of its s_k x s_k grid; off_j = sum_{i<j} n_i; L_k = sum_{i<=k} n_i.
+ * Step k (1-based): queries are the n_k tokens of scale k, keys/values are rows
+ * [0, L_k) of the cache, so the step-k attention map is [n_k, L_k].
+ *
+ * General rules.  No call throws, aborts or traps.  Every call returns a status; output
+ * arguments are written only on LITEVAR_OK.  "host" / "device" below say where a pointer
+ * must live.  Tensors passed to litevar_attn_forward are borrowed for the duration of the
+ * asynchronous work; the plan owns everything it allocates.
+ */
+#ifndef LITEVAR_H_
+#define LITEVAR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct litevar_plan litevar_plan_t; /* opaque; owns its device buffers */
+
+typedef enum {
+  LITEVAR_OK = 0,
+  LITEVAR_ERR_INVALID_ARG = 1,    /* NULL pointer, size or index out of range, misaligned tensor */
+  LITEVAR_ERR_UNSUPPORTED = 2,    /* valid request that this build does not implement */
+  LITEVAR_ERR_EMPTY_ROW = 3,      /* the window table leaves some query with no live key */
+  LITEVAR_ERR_ARCH = 4,           /* current device is not compute capability 10.x */
+  LITEVAR_ERR_OOM = 5,            /* device or host allocation failed */
+  LITEVAR_ERR_CUDA = 6,           /* a CUDA runtime/driver call failed */
+  LITEVAR_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait expired (see poll) */
+} litevar_status_t;
+
+/* Window shapes.  SQUARE: key (r',c') of scale j is live for query (r,c) of scale k iff
+ * |r' - ctr_j(r)| <= w and |c' - ctr_j(c)| <= w with ctr_j(x) = floor((2x+1) s_j / (2 s_k)),
+ * clipped at the grid border (the local window of paper Section 2 / Fig. 2(a), read as a 2-D
+ * neighbourhood of the co-located key cell).  BAND: key token t' of scale j is live iff
+ * |t' - floor((2q+1) n_j / (2 n_k))| <= w, the literal 1-D band about the part's diagonal in
+ * the flattened attention map. */
+enum { LITEVAR_WINDOW_SQUARE = 0, LITEVAR_WINDOW_BAND = 1 };
+
+/* Window specification (paper Section 2: one window width per part of the step-k map; the
+ * first parts stay global, "MDWA implementation details"). */
+typedef struct {
+  int32_t shape;            /* LITEVAR_WINDOW_SQUARE or LITEVAR_WINDOW_BAND */
+  int32_t n_global_scales;  /* key scales j <= this are fully live (paper: the merged first part, 3) */
+  int32_t rho_num, rho_den; /* default rule when radius == NULL: w_j = floor((2*num*s_j + den) / (2*den)),
+                               i.e. rho * s_j rounded half up (SQUARE) or rho * n_j (BAND) */
+  const int32_t* radius;    /* optional host table [n_sets][n_scales][n_scales], entry (set, k-1, j-1);
+                               -1 = whole part live; copied at plan time; entries with j > k ignored */
+  int32_t n_sets;           /* number of window tables (paper: widths are chosen per head); >= 1 */
+  const int32_t* head_to_set; /* host [n_heads], values in [0, n_sets); NULL = all heads use set 0 */
+} litevar_window_t;
+
+/* CFG sharing (paper Section 3): at a shared step the unconditional half of the batch
+ * receives a copy of the conditional half's attention output and is not computed. */
+typedef struct {
+  const uint8_t* share_step; /* host [n_scales], 1 = share at that step; NULL = never */
+} litevar_cfg_share_t;
+
+/* Element strides of a [2B, H, tokens, head_dim] tensor; head_dim has stride 1. */
+typedef struct {
+  int64_t batch, head, token;
+} litevar_strides_t;
+
+/* Forward kernel selection (testing / measurement). */
+enum {
+  LITEVAR_KERNEL_AUTO = 0,   /* tensor-core kernel for every step */
+  LITEVAR_KERNEL_SIMT = 1,   /* plain CUDA-core kernel (slow; cross-check and bring-up) */
+  LITEVAR_KERNEL_TCGEN05 = 2 /* tcgen05/TMEM/TMA kernel */
+};
+
+/*
+ * Build the per-step tile plan on the device (paper Section 2: parts, windows, global parts).
+ *
+ *   scales     host [n_scales], each in [1, 256]; n_scales in [1, 16]
+ *   n_heads    >= 1;  head_dim must be 64 (else UNSUPPORTED)
+ *   sm_scale   softmax scale; <= 0 selects 1/sqrt(head_dim)
+ *   window     host, required
+ *   share      host, may be NULL (no sharing)
+ *   stream     cudaStream_t the planner kernels run on (NULL = default stream); the call
+ *              synchronises that stream before it returns
+ *   out_plan   receives the plan; destroy with litevar_plan_destroy
+ *
+ * Device work: window table (radius per step and key scale), per-axis bounds
+ * [lo, hi] of every query row/column in every key scale, classification of every
+ * (query tile, key tile) pair as dead / partial / full, and compaction into a per-step
+ * CSR list in canonical order (query tile ascending, then key tile ascending), plus a
+ * 128x128-bit element mask for every partial pair.
+ * Errors: INVALID_ARG, UNSUPPORTED, EMPTY_ROW, ARCH, OOM, CUDA.
+ */
+litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int32_t n_heads,
+                                   int32_t head_dim, float sm_scale, const litevar_window_t* window,
+                                   const litevar_cfg_share_t* share, void* stream,
+                                   litevar_plan_t** out_plan);
+
+/*
+ * Step-k attention (paper Section 2 for the mask, Section 3 for sharing):
+ *   out[b,h,q,:] = sum_{t live} softmax_t(sm_scale * Q[b,h,q,:] . K[b,h,t,:]) V[b,h,t,:]
+ * for b in [0, 2B), h in [0, H), q in [0, n_k), t in [0, L_k); scores and sums in fp32,
+ * probabilities rounded to bf16 for the PV product, output rounded to bf16.
+ *
+ *   step_k       1-based step
+ *   batch_pairs  B; tensors hold 2B batch rows, rows [0,B) conditional, [B,2B) unconditional
+ *   Q, out       device bf16 [2B, H, n_k, 64] with the given strides
+ *   Kcache,Vcache device bf16 [2B, H, >= L_k, 64]; only rows [0, L_k) are read
+ *   strides      in elements; each a multiple of 8; base pointers 16-byte aligned
+ *   stream       cudaStream_t; the call is asynchronous, allocates nothing, synchronises nothing
+ *
+ * At a shared step the kernel runs for rows [0,B) only, never reads rows [B,2B) of Q/K/V,
+ * and stores every output tile to rows b and b+B.  Every element of out[0..2B)[h][0..n_k)
+ * is written.  Errors: INVALID_ARG (before any launch), CUDA.
+ */
+litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
+                                      const void* Q, const litevar_strides_t* sq,
+                                      const void* Kcache, const litevar_strides_t* sk,
+                                      const void* Vcache, const litevar_strides_t* sv,
+                                      void* out, const litevar_strides_t* so, void* stream);
+
+/* Counts for step k and window set `set`: live map entries, live / full / partial tile pairs. */
+litevar_status_t litevar_plan_stats(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                    int64_t* live_entries, int64_t* live_tiles, int64_t* full_tiles,
+                                    int64_t* partial_tiles);
+
+/* Sizes of the step-k tile plan of one window set. */
+litevar_status_t litevar_plan_tile_counts(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                          int32_t* n_q_tiles, int32_t* n_key_tiles, int32_t* n_pairs);
+
+/*
+ * Copy the step-k tile plan to host arrays sized from litevar_plan_tile_counts (any may be NULL):
+ *   q_tile_geom   [n_q_tiles][4]   {first token, slots, row stride, columns}: slot m is token
+ *                                  first + (m / columns) * row_stride + (m % columns)
+ *   key_tile_geom [n_key_tiles][4] same, tokens index the K/V cache
+ *   row_ptr       [n_q_tiles + 1]  CSR offsets into the pair arrays
+ *   pair_key_tile [n_pairs]        key tile of each live pair, ascending inside a query tile
+ *   pair_is_full  [n_pairs]        1 = every slot pair live (no element mask), 0 = partial
+ */
+litevar_status_t litevar_plan_export_tiles(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                           int32_t* q_tile_geom, int32_t* key_tile_geom,
+                                           int32_t* row_ptr, int32_t* pair_key_tile,
+                                           uint8_t* pair_is_full);
+
+/* Copy the window radii of step k (host out [n_scales], -1 = global, entries j > k are -1) and the
+ * per-axis bounds the device computed (host out [step_k][s_k][2] int32: lo, hi of query row or
+ * column x in key scale j; SQUARE windows only; either pointer may be NULL). */
+litevar_status_t litevar_plan_export_bounds(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                            int32_t* radius, int32_t* bounds);
+
+/* Expand the tile list and element masks of step k into a dense bit mask on the device:
+ * dev_bits is n_k rows of ceil(L_k / 32) uint32 words, bit (t & 31) of word t >> 5 = live(q, t).
+ * Runs on `stream`, asynchronous.  The mask blocks read here are the ones the attention kernel reads. */
+litevar_status_t litevar_plan_materialize_mask(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                               void* dev_bits, void* stream);
+
+/* Synchronises the device and reports LITEVAR_ERR_DEVICE_TIMEOUT if any forward kernel launched
+ * with this plan gave up on a bounded wait since the last poll (the flag is then cleared). */
+litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan);
+
+/* Select the forward kernel (LITEVAR_KERNEL_*).  Not thread-safe against concurrent forwards. */
+litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel);
+
+/* Frees the plan and its device buffers.  NULL is allowed. */
+void litevar_plan_destroy(litevar_plan_t* plan);
+
+/* Static string for a status code. */
+const char* litevar_status_string(litevar_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LITEVAR_H_ */

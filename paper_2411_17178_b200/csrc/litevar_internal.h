@@ -1,0 +1,96 @@
+// Internal definitions shared by the translation units of liblitevar (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "litevar.h"
+
+namespace litevar {
+
+constexpr int kMaxScales = 16;
+constexpr int kMaxScale = 256;
+constexpr int kHeadDim = 64;
+constexpr int kBlockM = 128;  // query slots per tile
+constexpr int kBlockN = 128;  // key slots per tile
+constexpr int kMaskWordsPerRow = kBlockN / 32;
+
+// Schedule of one plan, passed to kernels by value (paper Section 2: n_k = s_k^2, off_j, L_k).
+struct Schedule {
+  int32_t n_scales;
+  int32_t scale[kMaxScales];
+  int32_t off[kMaxScales + 1];  // off[j] = tokens before scale j+1 (0-based j); off[K] = total
+};
+
+// One live (query tile, key tile) pair: key tile index and index of its 128x128-bit mask block
+// (-1: every slot pair is live, no element mask).
+struct Pair {
+  int32_t key_tile;
+  int32_t mask_block;
+};
+
+// Device-visible tile plan of one (step, window set).
+struct SetDesc {
+  const int32_t* row_ptr;  // [n_q_tiles + 1]
+  const Pair* pairs;       // [n_pairs]
+  const uint4* mask;       // [n_partial][kBlockM] : 128 key bits per query slot
+};
+
+struct StepSet {
+  int32_t n_pairs = 0, n_partial = 0, n_full = 0;
+  int64_t live_entries = 0;
+  int32_t* d_row_ptr = nullptr;
+  Pair* d_pairs = nullptr;
+  uint4* d_mask = nullptr;
+  int2* d_bounds = nullptr;  // [k][s_k] {lo, hi} per key scale and query row/column (SQUARE)
+};
+
+struct Step {
+  int32_t s_k = 0, n_k = 0, L_k = 0, n_q_tiles = 0, n_key_tiles = 0;
+  bool share = false;
+  std::vector<StepSet> sets;
+  SetDesc* d_sets = nullptr;  // [n_sets]
+};
+
+// Arguments of one forward launch, common to both kernels.
+struct FwdParams {
+  const SetDesc* sets;          // [n_sets] for this step
+  const int32_t* head_to_set;   // [H] or nullptr (all heads use set 0)
+  const uint16_t* q;
+  const uint16_t* k;
+  const uint16_t* v;
+  uint16_t* out;
+  int64_t q_sb, q_sh, q_st;     // element strides: batch, head, token
+  int64_t k_sb, k_sh, k_st;
+  int64_t v_sb, v_sh, v_st;
+  int64_t o_sb, o_sh, o_st;
+  int32_t n_k, L_k, n_heads;
+  int32_t batch_computed;       // rows the grid covers (B when shared, else 2B)
+  int32_t share_offset;         // B when the step is shared (second store at row b + B), else 0
+  float sm_scale;
+  int32_t* status;              // device word, set non-zero when a bounded wait expires
+};
+
+cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
+
+// Tensor-core path.  Returns LITEVAR_OK or an error status (tensor-map encoding can fail).
+litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
+
+}  // namespace litevar
+
+struct litevar_plan {
+  litevar::Schedule sched;
+  int32_t n_heads = 0, n_sets = 1, shape = 0, n_global = 0, rho_num = 1, rho_den = 4;
+  float sm_scale = 0.125f;
+  int32_t kernel = LITEVAR_KERNEL_AUTO;
+  int device = 0;
+  std::vector<int32_t> radius;        // [n_sets][K][K]
+  std::vector<int32_t> head_to_set;   // [H] (empty when n_sets == 1)
+  int32_t* d_head_to_set = nullptr;
+  int32_t* d_radius = nullptr;        // [n_sets][K][K]
+  int32_t* d_status = nullptr;
+  std::vector<litevar::Step> steps;   // [K]
+  std::vector<void*> allocations;     // every cudaMalloc of the plan
+};

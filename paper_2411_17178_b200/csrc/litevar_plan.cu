@@ -1,0 +1,630 @@
+// Host side of the C ABI and the device-side mask planner.
+//
+// The planner turns the window definition of the paper's Section 2 (one window per part of the
+// step-k attention map, the first parts global) into, per step, a CSR list of live
+// (query tile, key tile) pairs plus a 128x128-bit element mask for every partially live pair.
+// Everything that depends on the mask geometry happens here; the attention kernels only walk
+// the list and apply the bit masks, so they are independent of the window shape.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "litevar_internal.h"
+
+using namespace litevar;
+
+namespace {
+
+#define LV_CUDA(expr)                          \
+  do {                                         \
+    cudaError_t e__ = (expr);                  \
+    if (e__ != cudaSuccess) {                  \
+      (void)cudaGetLastError();                \
+      return e__ == cudaErrorMemoryAllocation ? LITEVAR_ERR_OOM : LITEVAR_ERR_CUDA; \
+    }                                          \
+  } while (0)
+
+// ------------------------------------------------------------------ A1: window table
+// radius[k][j] for step k+1 and key scale j+1 (0-based indices here); -1 = whole part live.
+// Default rule: scales j <= n_global are global; otherwise round-half-up of rho * s_j (SQUARE)
+// or rho * n_j (BAND).  A caller table is copied, with unused entries (j > k) set to -1.
+__global__ void window_table_kernel(Schedule sc, int shape, int n_global, int rho_num, int rho_den,
+                                    const int32_t* user, int32_t* radius) {
+  int K = sc.n_scales;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < K * K; i += gridDim.x * blockDim.x) {
+    int k = i / K, j = i % K;
+    int w;
+    if (j > k) {
+      w = -1;
+    } else if (user != nullptr) {
+      w = user[i] < 0 ? -1 : user[i];
+    } else if (j < n_global) {
+      w = -1;
+    } else {
+      long long ext = shape == LITEVAR_WINDOW_BAND ? (long long)sc.scale[j] * sc.scale[j] : sc.scale[j];
+      w = (int)((2LL * rho_num * ext + rho_den) / (2LL * rho_den));
+    }
+    radius[i] = w;
+  }
+}
+
+// ------------------------------------------------------------------ A2: per-axis bounds
+// For query row (or column) x of scale k and key scale j: the key cell containing the centre of
+// cell x is ctr = floor((2x+1) s_j / (2 s_k)); the live interval is [ctr-w, ctr+w] clipped to the grid.
+__global__ void bounds_kernel(Schedule sc, int k0, const int32_t* radius_row, int2* bounds) {
+  int s_k = sc.scale[k0];
+  int total = (k0 + 1) * s_k;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    int j = i / s_k, x = i % s_k;
+    int s_j = sc.scale[j];
+    int w = radius_row[j];
+    int2 b;
+    if (w < 0) {
+      b = make_int2(0, s_j - 1);
+    } else {
+      int ctr = ((2 * x + 1) * s_j) / (2 * s_k);
+      b = make_int2(max(0, ctr - w), min(s_j - 1, ctr + w));
+    }
+    bounds[i] = b;
+  }
+}
+
+// ------------------------------------------------------------------ element predicate over one tile pair
+struct TileGeom {
+  int k0;           // 0-based step
+  int s_k, n_k, L_k;
+  int n_key_tiles;
+  int shape;
+};
+
+// Live bits of query slot `m` of query tile `qt` against the 128 key slots of key tile `kt`.
+// Must be called by all 128 threads of the block (fills shared key-slot tables).
+__device__ uint4 tile_row_bits(const Schedule& sc, const TileGeom& g, const int2* __restrict__ bounds,
+                               const int32_t* __restrict__ radius_row, int qt, int kt,
+                               int16_t* ks_j, int16_t* ks_r, int16_t* ks_c, int32_t* ks_t) {
+  int m = threadIdx.x;
+  {
+    int t = kt * kBlockN + m;  // raster key tiles: slot n of tile kt is cache row kt*128 + n
+    int j = -1, r = 0, c = 0, tin = 0;
+    if (t < g.L_k) {
+      j = 0;
+      while (t >= sc.off[j + 1]) ++j;
+      tin = t - sc.off[j];
+      r = tin / sc.scale[j];
+      c = tin % sc.scale[j];
+    }
+    ks_j[m] = (int16_t)j;
+    ks_r[m] = (int16_t)r;
+    ks_c[m] = (int16_t)c;
+    ks_t[m] = tin;
+  }
+  __syncthreads();
+  int q = qt * kBlockM + m;
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  if (q < g.n_k) {
+    int r = q / g.s_k, c = q % g.s_k;
+    int cur_j = -2;
+    int2 br = make_int2(0, -1), bc = make_int2(0, -1);
+    long long band_ctr = 0;
+    int band_w = -1;
+    for (int n = 0; n < kBlockN; ++n) {
+      int j = ks_j[n];
+      bool lv = false;
+      if (j >= 0) {
+        if (j != cur_j) {
+          cur_j = j;
+          if (g.shape == LITEVAR_WINDOW_SQUARE) {
+            br = bounds[j * g.s_k + r];
+            bc = bounds[j * g.s_k + c];
+          } else {
+            band_w = radius_row[j];
+            long long n_j = (long long)sc.scale[j] * sc.scale[j];
+            band_ctr = ((2LL * q + 1) * n_j) / (2LL * g.n_k);
+          }
+        }
+        if (g.shape == LITEVAR_WINDOW_SQUARE) {
+          int kr = ks_r[n], kc = ks_c[n];
+          lv = kr >= br.x && kr <= br.y && kc >= bc.x && kc <= bc.y;
+        } else {
+          long long d = (long long)ks_t[n] - band_ctr;
+          lv = band_w < 0 || (d <= band_w && -d <= band_w);
+        }
+      }
+      if (lv) w[n >> 5] |= 1u << (n & 31);
+    }
+  }
+  __syncthreads();
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// ------------------------------------------------------------------ A3 pass 1: classify every candidate pair
+// cls: 0 dead, 1 partial, 2 full (every valid query slot sees all 128 key slots live).
+__global__ void __launch_bounds__(128) classify_kernel(Schedule sc, TileGeom g, const int2* bounds,
+                                                       const int32_t* radius_row, uint8_t* cls,
+                                                       int32_t* row_live, unsigned long long* live_entries) {
+  __shared__ int16_t ks_j[kBlockN], ks_r[kBlockN], ks_c[kBlockN];
+  __shared__ int32_t ks_t[kBlockN];
+  int kt = blockIdx.x, qt = blockIdx.y;
+  uint4 b = tile_row_bits(sc, g, bounds, radius_row, qt, kt, ks_j, ks_r, ks_c, ks_t);
+  int q = qt * kBlockM + threadIdx.x;
+  bool valid = q < g.n_k;
+  int cnt = __popc(b.x) + __popc(b.y) + __popc(b.z) + __popc(b.w);
+  int any = __syncthreads_or(cnt != 0);
+  int all = __syncthreads_and(!valid || cnt == kBlockN);
+  if (valid && cnt) atomicAdd(&row_live[q], cnt);
+  // block total
+  for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if ((threadIdx.x & 31) == 0 && cnt) atomicAdd(live_entries, (unsigned long long)cnt);
+  if (threadIdx.x == 0) cls[qt * g.n_key_tiles + kt] = any ? (all ? 2 : 1) : 0;
+}
+
+// ------------------------------------------------------------------ A3 pass 2: count + exclusive scan
+// One block; thread qt counts the live and partial pairs of query tile qt, then a serial scan
+// (at most 512 tiles) writes the CSR offsets.  totals = {pairs, partial, full}.
+__global__ void count_scan_kernel(int n_q_tiles, int n_key_tiles, const uint8_t* cls, int32_t* row_ptr,
+                                  int32_t* partial_base, int32_t* totals) {
+  extern __shared__ int32_t sh[];
+  int32_t* nl = sh;
+  int32_t* np = sh + n_q_tiles;
+  for (int qt = threadIdx.x; qt < n_q_tiles; qt += blockDim.x) {
+    int l = 0, p = 0;
+    for (int kt = 0; kt < n_key_tiles; ++kt) {
+      int c = cls[qt * n_key_tiles + kt];
+      l += c != 0;
+      p += c == 1;
+    }
+    nl[qt] = l;
+    np[qt] = p;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int al = 0, ap = 0;
+    for (int qt = 0; qt < n_q_tiles; ++qt) {
+      row_ptr[qt] = al;
+      partial_base[qt] = ap;
+      al += nl[qt];
+      ap += np[qt];
+    }
+    row_ptr[n_q_tiles] = al;
+    totals[0] = al;
+    totals[1] = ap;
+    totals[2] = al - ap;
+  }
+}
+
+// ------------------------------------------------------------------ A3 pass 3: compact in canonical order
+__global__ void compact_kernel(int n_q_tiles, int n_key_tiles, const uint8_t* cls, const int32_t* row_ptr,
+                               const int32_t* partial_base, Pair* pairs, int32_t* mask_block_of) {
+  int qt = blockIdx.x * blockDim.x + threadIdx.x;
+  if (qt >= n_q_tiles) return;
+  int o = row_ptr[qt], pb = partial_base[qt];
+  for (int kt = 0; kt < n_key_tiles; ++kt) {
+    int c = cls[qt * n_key_tiles + kt];
+    int blk = -1;
+    if (c == 1) blk = pb++;
+    mask_block_of[qt * n_key_tiles + kt] = blk;
+    if (c != 0) {
+      pairs[o].key_tile = kt;
+      pairs[o].mask_block = blk;
+      ++o;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ A3 pass 4: element masks of partial pairs
+__global__ void __launch_bounds__(128) mask_bits_kernel(Schedule sc, TileGeom g, const int2* bounds,
+                                                        const int32_t* radius_row, const int32_t* mask_block_of,
+                                                        uint4* mask) {
+  __shared__ int16_t ks_j[kBlockN], ks_r[kBlockN], ks_c[kBlockN];
+  __shared__ int32_t ks_t[kBlockN];
+  int kt = blockIdx.x, qt = blockIdx.y;
+  int blk = mask_block_of[qt * g.n_key_tiles + kt];
+  if (blk < 0) return;  // uniform per block
+  uint4 b = tile_row_bits(sc, g, bounds, radius_row, qt, kt, ks_j, ks_r, ks_c, ks_t);
+  mask[(size_t)blk * kBlockM + threadIdx.x] = b;
+}
+
+__global__ void empty_row_kernel(int n_k, const int32_t* row_live, int32_t* flag) {
+  int q = blockIdx.x * blockDim.x + threadIdx.x;
+  if (q < n_k && row_live[q] == 0) atomicExch(flag, 1);
+}
+
+// ------------------------------------------------------------------ debug: dense mask from the tile plan
+__global__ void __launch_bounds__(128) materialize_kernel(SetDesc sd, int n_k, int L_k, uint32_t* dense) {
+  int qt = blockIdx.x, m = threadIdx.x;
+  int q = qt * kBlockM + m;
+  if (q >= n_k) return;
+  int words = (L_k + 31) / 32;
+  for (int p = sd.row_ptr[qt]; p < sd.row_ptr[qt + 1]; ++p) {
+    Pair pr = sd.pairs[p];
+    uint4 b = pr.mask_block < 0 ? make_uint4(~0u, ~0u, ~0u, ~0u)
+                                : sd.mask[(size_t)pr.mask_block * kBlockM + m];
+    uint32_t w[4] = {b.x, b.y, b.z, b.w};
+    int w0 = pr.key_tile * kMaskWordsPerRow;
+    for (int i = 0; i < 4; ++i)
+      if (w0 + i < words) dense[(size_t)q * words + w0 + i] = w[i];
+  }
+}
+
+template <typename T>
+litevar_status_t dev_alloc(litevar_plan* plan, T** out, size_t count) {
+  void* p = nullptr;
+  size_t bytes = count * sizeof(T);
+  if (bytes == 0) bytes = sizeof(T);
+  cudaError_t e = cudaMalloc(&p, bytes);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? LITEVAR_ERR_OOM : LITEVAR_ERR_CUDA;
+  }
+  plan->allocations.push_back(p);
+  *out = static_cast<T*>(p);
+  return LITEVAR_OK;
+}
+
+struct Scratch {
+  std::vector<void*> ptrs;
+  ~Scratch() {
+    for (void* p : ptrs) cudaFree(p);
+  }
+  template <typename T>
+  cudaError_t get(T** out, size_t count) {
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, count * sizeof(T) ? count * sizeof(T) : sizeof(T));
+    if (e == cudaSuccess) {
+      ptrs.push_back(p);
+      *out = static_cast<T*>(p);
+    }
+    return e;
+  }
+};
+
+litevar_status_t plan_step_set(litevar_plan* plan, int k0, int set, cudaStream_t stream) {
+  Step& st = plan->steps[k0];
+  StepSet& ss = st.sets[set];
+  const Schedule& sc = plan->sched;
+  const int K = sc.n_scales;
+  const int32_t* d_radius_row = plan->d_radius + ((size_t)set * K + k0) * K;
+
+  litevar_status_t s = dev_alloc(plan, &ss.d_bounds, (size_t)(k0 + 1) * st.s_k);
+  if (s != LITEVAR_OK) return s;
+  bounds_kernel<<<(unsigned)(((k0 + 1) * st.s_k + 255) / 256), 256, 0, stream>>>(sc, k0, d_radius_row, ss.d_bounds);
+
+  TileGeom g{k0, st.s_k, st.n_k, st.L_k, st.n_key_tiles, plan->shape};
+  Scratch tmp;
+  uint8_t* d_cls = nullptr;
+  int32_t *d_row_live = nullptr, *d_partial_base = nullptr, *d_totals = nullptr, *d_blk = nullptr;
+  unsigned long long* d_live = nullptr;
+  size_t n_cand = (size_t)st.n_q_tiles * st.n_key_tiles;
+  LV_CUDA(tmp.get(&d_cls, n_cand));
+  LV_CUDA(tmp.get(&d_row_live, (size_t)st.n_k));
+  LV_CUDA(tmp.get(&d_partial_base, (size_t)st.n_q_tiles));
+  LV_CUDA(tmp.get(&d_totals, 4));
+  LV_CUDA(tmp.get(&d_blk, n_cand));
+  LV_CUDA(tmp.get(&d_live, 1));
+  LV_CUDA(cudaMemsetAsync(d_row_live, 0, sizeof(int32_t) * st.n_k, stream));
+  LV_CUDA(cudaMemsetAsync(d_totals, 0, sizeof(int32_t) * 4, stream));
+  LV_CUDA(cudaMemsetAsync(d_live, 0, sizeof(unsigned long long), stream));
+
+  s = dev_alloc(plan, &ss.d_row_ptr, (size_t)st.n_q_tiles + 1);
+  if (s != LITEVAR_OK) return s;
+
+  dim3 grid2((unsigned)st.n_key_tiles, (unsigned)st.n_q_tiles);
+  classify_kernel<<<grid2, 128, 0, stream>>>(sc, g, ss.d_bounds, d_radius_row, d_cls, d_row_live, d_live);
+  empty_row_kernel<<<(unsigned)((st.n_k + 255) / 256), 256, 0, stream>>>(st.n_k, d_row_live, d_totals + 3);
+  int threads = st.n_q_tiles < 32 ? 32 : (st.n_q_tiles > 512 ? 512 : ((st.n_q_tiles + 31) / 32) * 32);
+  count_scan_kernel<<<1, threads, 2 * sizeof(int32_t) * st.n_q_tiles, stream>>>(
+      st.n_q_tiles, st.n_key_tiles, d_cls, ss.d_row_ptr, d_partial_base, d_totals);
+  int32_t totals[4];
+  unsigned long long live = 0;
+  LV_CUDA(cudaMemcpyAsync(totals, d_totals, sizeof(totals), cudaMemcpyDeviceToHost, stream));
+  LV_CUDA(cudaMemcpyAsync(&live, d_live, sizeof(live), cudaMemcpyDeviceToHost, stream));
+  LV_CUDA(cudaStreamSynchronize(stream));
+  if (totals[3] != 0) return LITEVAR_ERR_EMPTY_ROW;
+  ss.n_pairs = totals[0];
+  ss.n_partial = totals[1];
+  ss.n_full = totals[2];
+  ss.live_entries = (int64_t)live;
+
+  s = dev_alloc(plan, &ss.d_pairs, (size_t)ss.n_pairs);
+  if (s != LITEVAR_OK) return s;
+  s = dev_alloc(plan, &ss.d_mask, (size_t)ss.n_partial * kBlockM);
+  if (s != LITEVAR_OK) return s;
+  compact_kernel<<<(unsigned)((st.n_q_tiles + 127) / 128), 128, 0, stream>>>(
+      st.n_q_tiles, st.n_key_tiles, d_cls, ss.d_row_ptr, d_partial_base, ss.d_pairs, d_blk);
+  mask_bits_kernel<<<grid2, 128, 0, stream>>>(sc, g, ss.d_bounds, d_radius_row, d_blk, ss.d_mask);
+  LV_CUDA(cudaGetLastError());
+  LV_CUDA(cudaStreamSynchronize(stream));  // scratch is freed when `tmp` goes out of scope
+  return LITEVAR_OK;
+}
+
+bool strides_ok(const litevar_strides_t* s) {
+  return s && s->batch >= 0 && s->head >= 0 && s->token >= kHeadDim && (s->batch % 8) == 0 &&
+         (s->head % 8) == 0 && (s->token % 8) == 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* litevar_status_string(litevar_status_t status) {
+  switch (status) {
+    case LITEVAR_OK: return "ok";
+    case LITEVAR_ERR_INVALID_ARG: return "invalid argument";
+    case LITEVAR_ERR_UNSUPPORTED: return "unsupported";
+    case LITEVAR_ERR_EMPTY_ROW: return "window table leaves a query with no live key";
+    case LITEVAR_ERR_ARCH: return "device is not compute capability 10.x";
+    case LITEVAR_ERR_OOM: return "out of memory";
+    case LITEVAR_ERR_CUDA: return "CUDA error";
+    case LITEVAR_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+void litevar_plan_destroy(litevar_plan_t* plan) {
+  if (!plan) return;
+  for (void* p : plan->allocations) cudaFree(p);
+  delete plan;
+}
+
+litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int32_t n_heads, int32_t head_dim,
+                                   float sm_scale, const litevar_window_t* window,
+                                   const litevar_cfg_share_t* share, void* stream_, litevar_plan_t** out_plan) {
+  if (!scales || !window || !out_plan) return LITEVAR_ERR_INVALID_ARG;
+  if (n_scales < 1 || n_scales > kMaxScales || n_heads < 1 || head_dim < 1) return LITEVAR_ERR_INVALID_ARG;
+  for (int i = 0; i < n_scales; ++i)
+    if (scales[i] < 1 || scales[i] > kMaxScale) return LITEVAR_ERR_INVALID_ARG;
+  if (window->shape != LITEVAR_WINDOW_SQUARE && window->shape != LITEVAR_WINDOW_BAND) return LITEVAR_ERR_INVALID_ARG;
+  if (window->n_sets < 1 || window->n_sets > 64) return LITEVAR_ERR_INVALID_ARG;
+  if (!window->radius && (window->rho_den <= 0 || window->rho_num < 0 || window->n_global_scales < 0))
+    return LITEVAR_ERR_INVALID_ARG;
+  if (!window->radius && window->n_sets != 1) return LITEVAR_ERR_INVALID_ARG;
+  if (window->head_to_set)
+    for (int h = 0; h < n_heads; ++h)
+      if (window->head_to_set[h] < 0 || window->head_to_set[h] >= window->n_sets) return LITEVAR_ERR_INVALID_ARG;
+  if (head_dim != kHeadDim) return LITEVAR_ERR_UNSUPPORTED;
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  LV_CUDA(cudaGetDevice(&dev));
+  LV_CUDA(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return LITEVAR_ERR_ARCH;
+
+  litevar_plan* plan = new (std::nothrow) litevar_plan();
+  if (!plan) return LITEVAR_ERR_OOM;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  plan->device = dev;
+  plan->n_heads = n_heads;
+  plan->n_sets = window->n_sets;
+  plan->shape = window->shape;
+  plan->n_global = window->n_global_scales;
+  plan->rho_num = window->rho_num;
+  plan->rho_den = window->rho_den;
+  plan->sm_scale = sm_scale > 0.f ? sm_scale : 0.125f;
+  Schedule& sc = plan->sched;
+  memset(&sc, 0, sizeof(sc));
+  sc.n_scales = n_scales;
+  for (int i = 0; i < n_scales; ++i) {
+    sc.scale[i] = scales[i];
+    sc.off[i + 1] = sc.off[i] + scales[i] * scales[i];
+  }
+  const int K = n_scales;
+
+  auto fail = [&](litevar_status_t s) {
+    litevar_plan_destroy(plan);
+    return s;
+  };
+  litevar_status_t s;
+  if ((s = dev_alloc(plan, &plan->d_status, 1)) != LITEVAR_OK) return fail(s);
+  if ((s = dev_alloc(plan, &plan->d_radius, (size_t)plan->n_sets * K * K)) != LITEVAR_OK) return fail(s);
+  if (cudaMemsetAsync(plan->d_status, 0, sizeof(int32_t), stream) != cudaSuccess) return fail(LITEVAR_ERR_CUDA);
+
+  // A1: window tables on the device (default rule, or the caller's table normalised)
+  int32_t* d_user = nullptr;
+  Scratch tmp;
+  if (window->radius) {
+    if (tmp.get(&d_user, (size_t)plan->n_sets * K * K) != cudaSuccess) return fail(LITEVAR_ERR_OOM);
+    if (cudaMemcpyAsync(d_user, window->radius, sizeof(int32_t) * plan->n_sets * K * K, cudaMemcpyHostToDevice,
+                        stream) != cudaSuccess)
+      return fail(LITEVAR_ERR_CUDA);
+  }
+  for (int set = 0; set < plan->n_sets; ++set)
+    window_table_kernel<<<1, 256, 0, stream>>>(sc, plan->shape, plan->n_global, plan->rho_num, plan->rho_den,
+                                               d_user ? d_user + (size_t)set * K * K : nullptr,
+                                               plan->d_radius + (size_t)set * K * K);
+  plan->radius.resize((size_t)plan->n_sets * K * K);
+  if (cudaMemcpyAsync(plan->radius.data(), plan->d_radius, sizeof(int32_t) * plan->radius.size(),
+                      cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return fail(LITEVAR_ERR_CUDA);
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return fail(LITEVAR_ERR_CUDA);
+
+  if (window->head_to_set && plan->n_sets > 1) {
+    plan->head_to_set.assign(window->head_to_set, window->head_to_set + n_heads);
+    if ((s = dev_alloc(plan, &plan->d_head_to_set, (size_t)n_heads)) != LITEVAR_OK) return fail(s);
+    if (cudaMemcpyAsync(plan->d_head_to_set, plan->head_to_set.data(), sizeof(int32_t) * n_heads,
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return fail(LITEVAR_ERR_CUDA);
+  }
+
+  plan->steps.resize(K);
+  for (int k0 = 0; k0 < K; ++k0) {
+    Step& st = plan->steps[k0];
+    st.s_k = sc.scale[k0];
+    st.n_k = st.s_k * st.s_k;
+    st.L_k = sc.off[k0 + 1];
+    st.n_q_tiles = (st.n_k + kBlockM - 1) / kBlockM;
+    st.n_key_tiles = (st.L_k + kBlockN - 1) / kBlockN;
+    st.share = share && share->share_step && share->share_step[k0] != 0;
+    st.sets.resize(plan->n_sets);
+    std::vector<SetDesc> descs(plan->n_sets);
+    for (int set = 0; set < plan->n_sets; ++set) {
+      if ((s = plan_step_set(plan, k0, set, stream)) != LITEVAR_OK) return fail(s);
+      descs[set] = SetDesc{st.sets[set].d_row_ptr, st.sets[set].d_pairs, st.sets[set].d_mask};
+    }
+    if ((s = dev_alloc(plan, &st.d_sets, (size_t)plan->n_sets)) != LITEVAR_OK) return fail(s);
+    if (cudaMemcpyAsync(st.d_sets, descs.data(), sizeof(SetDesc) * plan->n_sets, cudaMemcpyHostToDevice,
+                        stream) != cudaSuccess)
+      return fail(LITEVAR_ERR_CUDA);
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return fail(LITEVAR_ERR_CUDA);
+  }
+  *out_plan = plan;
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
+                                      const void* Q, const litevar_strides_t* sq, const void* Kc,
+                                      const litevar_strides_t* sk, const void* Vc, const litevar_strides_t* sv,
+                                      void* out, const litevar_strides_t* so, void* stream_) {
+  if (!plan || !Q || !Kc || !Vc || !out) return LITEVAR_ERR_INVALID_ARG;
+  if (step_k < 1 || step_k > plan->sched.n_scales || batch_pairs < 1) return LITEVAR_ERR_INVALID_ARG;
+  if (!strides_ok(sq) || !strides_ok(sk) || !strides_ok(sv) || !strides_ok(so)) return LITEVAR_ERR_INVALID_ARG;
+  if (((uintptr_t)Q | (uintptr_t)Kc | (uintptr_t)Vc | (uintptr_t)out) & 15) return LITEVAR_ERR_INVALID_ARG;
+  const Step& st = plan->steps[step_k - 1];
+  FwdParams p;
+  p.sets = st.d_sets;
+  p.head_to_set = plan->n_sets > 1 ? plan->d_head_to_set : nullptr;
+  p.q = static_cast<const uint16_t*>(Q);
+  p.k = static_cast<const uint16_t*>(Kc);
+  p.v = static_cast<const uint16_t*>(Vc);
+  p.out = static_cast<uint16_t*>(out);
+  p.q_sb = sq->batch; p.q_sh = sq->head; p.q_st = sq->token;
+  p.k_sb = sk->batch; p.k_sh = sk->head; p.k_st = sk->token;
+  p.v_sb = sv->batch; p.v_sh = sv->head; p.v_st = sv->token;
+  p.o_sb = so->batch; p.o_sh = so->head; p.o_st = so->token;
+  p.n_k = st.n_k;
+  p.L_k = st.L_k;
+  p.n_heads = plan->n_heads;
+  p.batch_computed = st.share ? batch_pairs : 2 * batch_pairs;
+  p.share_offset = st.share ? batch_pairs : 0;
+  p.sm_scale = plan->sm_scale;
+  p.status = plan->d_status;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (plan->kernel == LITEVAR_KERNEL_SIMT) {
+    cudaError_t e = launch_forward_simt(p, st.n_q_tiles, stream);
+    if (e != cudaSuccess) {
+      (void)cudaGetLastError();
+      return LITEVAR_ERR_CUDA;
+    }
+    return LITEVAR_OK;
+  }
+  return launch_forward_tcgen05(p, st.n_q_tiles, stream);
+}
+
+static litevar_status_t check_step_set(const litevar_plan_t* plan, int32_t step_k, int32_t set) {
+  if (!plan || step_k < 1 || step_k > plan->sched.n_scales || set < 0 || set >= plan->n_sets)
+    return LITEVAR_ERR_INVALID_ARG;
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_stats(const litevar_plan_t* plan, int32_t step_k, int32_t set, int64_t* live_entries,
+                                    int64_t* live_tiles, int64_t* full_tiles, int64_t* partial_tiles) {
+  litevar_status_t s = check_step_set(plan, step_k, set);
+  if (s != LITEVAR_OK) return s;
+  const StepSet& ss = plan->steps[step_k - 1].sets[set];
+  if (live_entries) *live_entries = ss.live_entries;
+  if (live_tiles) *live_tiles = ss.n_pairs;
+  if (full_tiles) *full_tiles = ss.n_full;
+  if (partial_tiles) *partial_tiles = ss.n_partial;
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_tile_counts(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                          int32_t* n_q_tiles, int32_t* n_key_tiles, int32_t* n_pairs) {
+  litevar_status_t s = check_step_set(plan, step_k, set);
+  if (s != LITEVAR_OK) return s;
+  const Step& st = plan->steps[step_k - 1];
+  if (n_q_tiles) *n_q_tiles = st.n_q_tiles;
+  if (n_key_tiles) *n_key_tiles = st.n_key_tiles;
+  if (n_pairs) *n_pairs = st.sets[set].n_pairs;
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_export_tiles(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                           int32_t* q_tile_geom, int32_t* key_tile_geom, int32_t* row_ptr,
+                                           int32_t* pair_key_tile, uint8_t* pair_is_full) {
+  litevar_status_t s = check_step_set(plan, step_k, set);
+  if (s != LITEVAR_OK) return s;
+  const Step& st = plan->steps[step_k - 1];
+  const StepSet& ss = st.sets[set];
+  if (q_tile_geom)
+    for (int i = 0; i < st.n_q_tiles; ++i) {
+      int first = i * kBlockM, slots = st.n_k - first < kBlockM ? st.n_k - first : kBlockM;
+      q_tile_geom[4 * i + 0] = first;
+      q_tile_geom[4 * i + 1] = slots;
+      q_tile_geom[4 * i + 2] = 0;
+      q_tile_geom[4 * i + 3] = slots;
+    }
+  if (key_tile_geom)
+    for (int i = 0; i < st.n_key_tiles; ++i) {
+      int first = i * kBlockN, slots = st.L_k - first < kBlockN ? st.L_k - first : kBlockN;
+      key_tile_geom[4 * i + 0] = first;
+      key_tile_geom[4 * i + 1] = slots;
+      key_tile_geom[4 * i + 2] = 0;
+      key_tile_geom[4 * i + 3] = slots;
+    }
+  LV_CUDA(cudaDeviceSynchronize());
+  if (row_ptr)
+    LV_CUDA(cudaMemcpy(row_ptr, ss.d_row_ptr, sizeof(int32_t) * (st.n_q_tiles + 1), cudaMemcpyDeviceToHost));
+  if ((pair_key_tile || pair_is_full) && ss.n_pairs > 0) {
+    std::vector<Pair> pairs(ss.n_pairs);
+    LV_CUDA(cudaMemcpy(pairs.data(), ss.d_pairs, sizeof(Pair) * ss.n_pairs, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < ss.n_pairs; ++i) {
+      if (pair_key_tile) pair_key_tile[i] = pairs[i].key_tile;
+      if (pair_is_full) pair_is_full[i] = pairs[i].mask_block < 0 ? 1 : 0;
+    }
+  }
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_export_bounds(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                            int32_t* radius, int32_t* bounds) {
+  litevar_status_t s = check_step_set(plan, step_k, set);
+  if (s != LITEVAR_OK) return s;
+  const int K = plan->sched.n_scales;
+  const Step& st = plan->steps[step_k - 1];
+  if (radius)
+    memcpy(radius, plan->radius.data() + ((size_t)set * K + (step_k - 1)) * K, sizeof(int32_t) * K);
+  if (bounds) {
+    LV_CUDA(cudaDeviceSynchronize());
+    LV_CUDA(cudaMemcpy(bounds, st.sets[set].d_bounds, sizeof(int2) * step_k * st.s_k, cudaMemcpyDeviceToHost));
+  }
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_materialize_mask(const litevar_plan_t* plan, int32_t step_k, int32_t set,
+                                               void* dev_bits, void* stream_) {
+  litevar_status_t s = check_step_set(plan, step_k, set);
+  if (s != LITEVAR_OK) return s;
+  if (!dev_bits) return LITEVAR_ERR_INVALID_ARG;
+  const Step& st = plan->steps[step_k - 1];
+  const StepSet& ss = st.sets[set];
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  size_t words = (size_t)((st.L_k + 31) / 32);
+  LV_CUDA(cudaMemsetAsync(dev_bits, 0, sizeof(uint32_t) * words * st.n_k, stream));
+  SetDesc sd{ss.d_row_ptr, ss.d_pairs, ss.d_mask};
+  materialize_kernel<<<(unsigned)st.n_q_tiles, 128, 0, stream>>>(sd, st.n_k, st.L_k,
+                                                                   static_cast<uint32_t*>(dev_bits));
+  LV_CUDA(cudaGetLastError());
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan) {
+  if (!plan) return LITEVAR_ERR_INVALID_ARG;
+  int32_t v = 0;
+  LV_CUDA(cudaDeviceSynchronize());
+  LV_CUDA(cudaMemcpy(&v, plan->d_status, sizeof(v), cudaMemcpyDeviceToHost));
+  if (v != 0) {
+    LV_CUDA(cudaMemset(plan->d_status, 0, sizeof(v)));
+    return LITEVAR_ERR_DEVICE_TIMEOUT;
+  }
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel) {
+  if (!plan || kernel < LITEVAR_KERNEL_AUTO || kernel > LITEVAR_KERNEL_TCGEN05) return LITEVAR_ERR_INVALID_ARG;
+  plan->kernel = kernel;
+  return LITEVAR_OK;
+}
+
+}  // extern "C"
