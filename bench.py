@@ -1,0 +1,584 @@
+#!/usr/bin/env python
+"""Benchmark of the LiteVAR attention path (multi-diagonal window mask + CFG sharing) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference] [--no-extras]
+
+A "step" is one pass of the whole hot path over one batch: one full generation's attention,
+i.e. every scale step of every layer of the chosen workload (for the single-call workloads 1 and
+5: one call).  Rank 0 prints ONE JSON line.  The headline workload is the full 10-step VAR-d16
+schedule at 256px (16 layers x 16 heads, batch 2x8, default window, CFG sharing everywhere).
+
+value            useful TFLOP/s: 256 FLOP per live map entry of every (batch row, head) the kernel
+                 computes (under CFG sharing: the conditional half), inputs resident in HBM,
+                 the generation's calls replayed from one CUDA graph
+e2e              the same metric through the per-call API with pinned HOST buffers: every call
+                 copies its Q and the new scale's K/V rows to the device and its output back
+roofline         HBM bound for this workload: compulsory bytes (Q + K/V prefix read once per
+                 computed (b, h), output written for all 2B rows) over the measured time
+cpu_baseline     the CPU fp64 oracle timed on this machine's host cores on a bounded sample
+all_configs      the five benchmark workloads, window and full-mask variants (unless --no-extras)
+
+With --impl reference the oracle itself is timed (rank 0 only) and printed in the same format.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2411_17178_b200 import workloads as wl  # noqa: E402
+
+FLOP_PER_ENTRY = 4 * wl.HEAD_DIM          # QK^T and PV, multiply + add, per live (q, t)
+TILE_FLOP = FLOP_PER_ENTRY * 128 * 128    # one executed 128x128 tile pair
+METRIC = "multi-diag attn useful TFLOP/s (live entries only)"
+UNIT = "TFLOP/s"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------- accounting
+def schedule_counts(plan, w: wl.Workload):
+    """Per step: live entries, executed tile pairs (from the plan), n_k, L_k."""
+    out = {}
+    for k in w.steps:
+        st = plan.stats(k)
+        out[k] = dict(live=st["live_entries"], tiles=st["live_tiles"], n_k=w.scales[k - 1] ** 2,
+                      L_k=wl.cache_len(w.scales, k))
+    return out
+
+
+def per_layer_work(w: wl.Workload, counts, share: bool):
+    """Useful FLOP, executed FLOP and compulsory HBM bytes of one layer's calls."""
+    rows = 2 * w.batch_pairs
+    computed = w.batch_pairs if share else rows
+    useful = executed = nbytes = 0
+    for k in w.steps:
+        c = counts[k]
+        useful += c["live"] * FLOP_PER_ENTRY * computed * w.n_heads
+        executed += c["tiles"] * TILE_FLOP * computed * w.n_heads
+        row_b = wl.HEAD_DIM * 2
+        nbytes += w.n_heads * (computed * (c["n_k"] + 2 * c["L_k"]) + rows * c["n_k"]) * row_b
+    return useful, executed, nbytes
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """nvidia-smi in a child process, one CSV line every 100 ms, for the GPU this rank uses."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.lines = []
+        try:
+            uuid = torch.cuda.get_device_properties(device_index).uuid
+            ident = "GPU-" + str(uuid) if not str(uuid).startswith("GPU-") else str(uuid)
+        except Exception:
+            ident = str(device_index)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", ident, "--query-gpu=timestamp," + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        self.lines = [l for l in out.splitlines() if l.strip()]
+        self.proc = None
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        # "under load": the upper half of the samples (idle samples before the first launch drop out)
+        hot = sorted(sm)[len(sm) // 2:]
+        return {"sm_mhz": statistics.median(hot), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------- GPU arm
+def device_randn_bf16(shape, seed, device):
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return torch.randn(*shape, generator=g, dtype=torch.float32, device=device).to(torch.bfloat16)
+
+
+class Buffers:
+    """Device tensors of `n_sets` layers of one workload (seeded, generated on the device)."""
+
+    def __init__(self, w: wl.Workload, n_sets: int, device):
+        rows = 2 * w.batch_pairs
+        L = wl.cache_len(w.scales, max(w.steps))
+        self.k, self.v, self.q, self.out = [], [], [], []
+        for layer in range(n_sets):
+            k = device_randn_bf16((rows, w.n_heads, L, wl.HEAD_DIM), wl.seed_for(w.index, layer, 0, 1), device)
+            if w.key_head_scale:
+                k = (k.float() * wl.head_scales(w.n_heads).to(device).view(1, -1, 1, 1)).to(torch.bfloat16)
+            self.k.append(k)
+            self.v.append(device_randn_bf16((rows, w.n_heads, L, wl.HEAD_DIM), wl.seed_for(w.index, layer, 0, 2),
+                                            device))
+            qs, outs = {}, {}
+            for step in w.steps:
+                n_k = w.scales[step - 1] ** 2
+                qs[step] = device_randn_bf16((rows, w.n_heads, n_k, wl.HEAD_DIM),
+                                             wl.seed_for(w.index, layer, step, 0), device)
+                outs[step] = torch.empty_like(qs[step])
+            self.q.append(qs)
+            self.out.append(outs)
+        self.n_sets = n_sets
+
+    def bytes(self):
+        tot = 0
+        for i in range(self.n_sets):
+            tot += self.k[i].numel() * 2 + self.v[i].numel() * 2
+            tot += sum(t.numel() * 4 for t in self.q[i].values())
+        return tot
+
+
+def sets_needed(w: wl.Workload, budget_bytes=3 << 30, min_bytes=400 << 20):
+    """Distinct layer buffer sets: all layers when they fit the budget, else as many as the budget
+    holds; at least enough that one pass over them exceeds the 126 MB L2 several times."""
+    rows = 2 * w.batch_pairs
+    L = wl.cache_len(w.scales, max(w.steps))
+    nq = sum(w.scales[s - 1] ** 2 for s in w.steps)
+    per = rows * w.n_heads * (2 * L + 2 * nq) * wl.HEAD_DIM * 2
+    need = max(1, -(-min_bytes // per))
+    n = max(need, min(w.n_layers, max(1, budget_bytes // per)))
+    return int(n), per
+
+
+def generation_calls(w: wl.Workload, n_sets: int, repeat_layers: int):
+    """(step, buffer set) for every call of one generation, step-major as a model runs them."""
+    return [(k, layer % n_sets) for k in w.steps for layer in range(repeat_layers)]
+
+
+def run_generation(plan, w, bufs, calls, stream=None):
+    for k, s in calls:
+        plan.forward(k, w.batch_pairs, bufs.q[s][k], bufs.k[s], bufs.v[s], bufs.out[s][k], stream=stream)
+
+
+def time_graph(plan, w, bufs, calls, steps, warmup, dist_barrier=None):
+    """Capture one generation in a CUDA graph; time `steps` replays with CUDA events."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run_generation(plan, w, bufs, calls)      # warm: function attributes, first-touch
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run_generation(plan, w, bufs, calls)
+    for _ in range(warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    if dist_barrier:
+        dist_barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist_barrier:
+        dist_barrier()
+    return e0.elapsed_time(e1) / steps   # ms per generation
+
+
+def time_eager(plan, w, bufs, calls, steps, warmup):
+    for _ in range(warmup):
+        run_generation(plan, w, bufs, calls)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        run_generation(plan, w, bufs, calls)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def time_e2e(plan, w: wl.Workload, steps, warmup, device):
+    """Per-call API with host buffers: H2D of the call's Q and of the new scale's K/V rows (only the
+    batch rows the call computes), forward, D2H of the call's output.  One layer's device cache is
+    reused for every layer (the copies and the calls are the same)."""
+    rows = 2 * w.batch_pairs
+    share = w.share_cfg
+    comp = w.batch_pairs if share else rows
+    L = wl.cache_len(w.scales, max(w.steps))
+    H, D = w.n_heads, wl.HEAD_DIM
+    host_k, host_v = wl.make_kv(w, 0)
+    host_q = {k: wl.make_q(w, 0, k).pin_memory() for k in w.steps}
+    host_out = {k: torch.empty_like(host_q[k]).pin_memory() for k in w.steps}
+    dk = torch.zeros((rows, H, L, D), dtype=torch.bfloat16, device=device)
+    dv = torch.zeros_like(dk)
+    dq = {k: torch.empty((rows, H, w.scales[k - 1] ** 2, D), dtype=torch.bfloat16, device=device) for k in w.steps}
+    do = {k: torch.empty_like(dq[k]) for k in w.steps}
+    off = [0]
+    for s in w.scales:
+        off.append(off[-1] + s * s)
+    if min(w.steps) > 1:  # single-step workloads: the earlier scales are already cached on the device
+        a = off[min(w.steps) - 1]
+        dk[:, :, :a].copy_(host_k[:, :, :a])
+        dv[:, :, :a].copy_(host_v[:, :, :a])
+    # the rows a call appends to the cache, contiguous in pinned host memory
+    new_k = {k: host_k[:comp, :, off[k - 1]:off[k]].contiguous().pin_memory() for k in w.steps}
+    new_v = {k: host_v[:comp, :, off[k - 1]:off[k]].contiguous().pin_memory() for k in w.steps}
+    h2d = d2h = 0
+    for k in w.steps:
+        n_k = w.scales[k - 1] ** 2
+        h2d += w.n_layers * comp * H * n_k * D * 2 * 3
+        d2h += w.n_layers * rows * H * n_k * D * 2
+
+    def generation():
+        for k in w.steps:
+            a, b = off[k - 1], off[k]
+            for _layer in range(w.n_layers):
+                dq[k][:comp].copy_(host_q[k][:comp], non_blocking=True)
+                dk[:comp, :, a:b].copy_(new_k[k], non_blocking=True)
+                dv[:comp, :, a:b].copy_(new_v[k], non_blocking=True)
+                plan.forward(k, w.batch_pairs, dq[k], dk, dv, do[k])
+                host_out[k].copy_(do[k], non_blocking=True)
+
+    for _ in range(warmup):
+        generation()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        generation()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps, h2d, d2h
+
+
+def make_plan(w: wl.Workload, variant: str, rho=None):
+    from paper_2411_17178_b200 import binding
+    share = [1] * len(w.scales) if w.share_cfg else None
+    if variant == "dense":
+        K = len(w.scales)
+        return binding.Plan(w.scales, n_heads=w.n_heads, radius=np.full((K, K), -1, np.int32), share_steps=share)
+    return binding.Plan(w.scales, n_heads=w.n_heads, rho=rho or w.rho, share_steps=share)
+
+
+def measure_config(w: wl.Workload, variant: str, rho, steps, warmup, device, pk, bufs=None):
+    plan = make_plan(w, variant, rho)
+    counts = schedule_counts(plan, w)
+    useful, executed, nbytes = per_layer_work(w, counts, w.share_cfg)
+    n_sets, per_set = sets_needed(w)
+    if bufs is None:
+        bufs = Buffers(w, n_sets, device)
+    n_sets = bufs.n_sets
+    repeat = max(w.n_layers, n_sets)           # single-call workloads rotate over the sets
+    calls = generation_calls(w, n_sets, repeat)
+    ms = time_graph(plan, w, bufs, calls, steps, warmup)
+    assert plan.poll() == 0, "device-side wait timed out"
+    scale = repeat / w.n_layers                # calls timed per generation's worth of calls
+    us_gen = ms * 1e3 / scale
+    res = dict(config=w.index, workload=w.name, variant=variant,
+               rho=list(rho or w.rho) if variant == "window" else None,
+               calls_per_generation=len(w.steps) * w.n_layers,
+               us_per_generation=round(us_gen, 2),
+               us_per_call=round(us_gen / (len(w.steps) * w.n_layers), 3),
+               useful_tflops=round(useful * w.n_layers / (us_gen * 1e-6) / 1e12, 2),
+               executed_tflops=round(executed * w.n_layers / (us_gen * 1e-6) / 1e12, 2),
+               live_density_in_tiles=round(useful / executed, 4),
+               useful_frac_of_bf16_peak=round(useful * w.n_layers / (us_gen * 1e-6) / 1e12 / pk["bf16"], 4),
+               hbm_gbs_compulsory=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9, 1),
+               hbm_frac=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9 / pk["hbm"], 4),
+               buffer_sets=n_sets)
+    plan.close()
+    return res, bufs
+
+
+def gpu_arm(args):
+    from paper_2411_17178_b200 import build as lvbuild
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the attention path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    barrier = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+        def barrier():
+            dist.barrier()
+            torch.cuda.synchronize()
+    if rank == 0:
+        lvbuild.build()
+    if barrier:
+        barrier()
+    pk = peaks()
+    w = wl.WORKLOADS[args.config]
+    variant = "dense" if args.dense else "window"
+
+    # ---- headline: K generations of the chosen workload, replicated on every rank (no collective:
+    # (batch row, head) units are independent, each rank holds its own batch)
+    plan = make_plan(w, variant, tuple(args.rho) if args.rho else None)
+    counts = schedule_counts(plan, w)
+    useful, executed, nbytes = per_layer_work(w, counts, w.share_cfg)
+    n_sets, per_set = sets_needed(w)
+    bufs = Buffers(w, n_sets, device)
+    repeat = max(w.n_layers, n_sets)
+    calls = generation_calls(w, n_sets, repeat)
+    scale = repeat / w.n_layers
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms = time_graph(plan, w, bufs, calls, args.steps, args.warmup, barrier)
+    if sampler:
+        # keep the GPU in the same state a little longer so that short runs still collect samples
+        t_end = time.time() + (0.0 if args.kernel_only else max(0.0, 1.0 - ms * args.steps / 1e3))
+        while time.time() < t_end:
+            run_generation(plan, w, bufs, calls)
+            torch.cuda.synchronize()
+        sampler.stop()
+    status = plan.poll()
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_step = ms / scale
+    gen_useful = useful * w.n_layers
+    value = world * gen_useful / (ms_step * 1e-3) / 1e12
+    launches_per_step = len(calls)
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    out = {
+        "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"config {w.index}: {w.name}", "variant": variant, "scales": list(w.scales),
+                   "steps_per_generation": len(w.steps), "layers": w.n_layers, "heads": w.n_heads,
+                   "batch": f"2x{w.batch_pairs}", "cfg_share": w.share_cfg, "window_rho": list(args.rho or w.rho),
+                   "launch": "one CUDA graph replay per generation",
+                   "l2": f"inputs larger than L2: {bufs.bytes() / 1e6:.0f} MB over {bufs.n_sets} layer buffer "
+                         "sets visited step-major"},
+        "gpu_launches": launches_per_step * args.steps,
+        "us_per_generation": round(ms_step * 1e3, 2),
+        "us_per_image": round(ms_step * 1e3 / w.batch_pairs, 2),
+        "cfg_effective_tflops": round(value * (2 if w.share_cfg else 1), 3),
+        "executed_tflops": round(world * executed * w.n_layers / (ms_step * 1e-3) / 1e12, 3),
+        "useful_frac_of_bf16_peak": round(value / world / pk["bf16"], 5),
+        "device_status": status,
+        "peaks": pk,
+    }
+    if sampler:
+        out["clocks"] = sampler.summary()
+
+    # ---- roofline of the forward kernel on this workload (the only kernel in the timed region)
+    alg_bytes_launch = nbytes * w.n_layers / (len(w.steps) * w.n_layers)
+    avg_launch_s = ms_step * 1e-3 / (len(w.steps) * w.n_layers)
+    achieved = alg_bytes_launch / avg_launch_s / 1e9
+    out["roofline"] = {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm"], "unit": "GB/s",
+                       "frac": round(achieved / pk["hbm"], 4), "traffic": None,
+                       "kernel": "fwd_tc_kernel", "peak_source": pk["source"],
+                       "algorithmic_bytes_per_launch": round(alg_bytes_launch),
+                       "avg_launch_us": round(avg_launch_s * 1e6, 3)}
+
+    if args.kernel_only:
+        plan.close()
+        print(json.dumps(out), flush=True)
+        return
+
+    # ---- eager per-call figure (ctypes call + tensor-map encoding per launch on the host)
+    eager_ms = time_eager(plan, w, bufs, calls, max(2, min(args.steps, 10)), 1) / scale
+    out["eager_us_per_generation"] = round(eager_ms * 1e3, 2)
+
+    # ---- end to end with host buffers
+    e2e_ms, h2d, d2h = time_e2e(plan, w, max(1, min(args.steps, 5)), 1, device)
+    out["e2e"] = {"value": round(gen_useful / (e2e_ms * 1e-3) / 1e12 * world, 4), "unit": UNIT,
+                  "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4)}
+    plan.close()
+    del bufs
+    torch.cuda.empty_cache()
+
+    # ---- CPU oracle baseline (rank 0, N = 1 only)
+    if world == 1 and not args.no_cpu:
+        out["cpu_baseline"] = oracle_baseline(w, args.cpu_seconds)
+
+    # ---- the five workloads, window and dense variants
+    if world == 1 and not args.no_extras:
+        table = []
+        reps, warm = 5, 3
+        for idx in (1, 2, 3, 4, 5):
+            wi = wl.WORKLOADS[idx]
+            shared_bufs = None
+            variants = [("window", r) for r in (wi.rho_sweep or (wi.rho,))] + [("dense", None)]
+            for var, rho in variants:
+                r, shared_bufs = measure_config(wi, var, rho, reps, warm, device, pk, shared_bufs)
+                table.append(r)
+            del shared_bufs
+            torch.cuda.empty_cache()
+        out["all_configs"] = table
+    print(json.dumps(out), flush=True)
+
+
+# --------------------------------------------------------------------------------------- CPU arm
+def oracle_sample(w: wl.Workload, seconds: float):
+    """Run the oracle, as it stands, over layers of the workload until `seconds` have passed.
+    Returns (useful FLOP done, elapsed s, description)."""
+    from oracle import litevar_oracle as orc
+    tab = orc.window_table(w.scales, rho=w.rho)
+    rows = 2 * w.batch_pairs
+    done_flop = 0.0
+    t0 = time.perf_counter()
+    what = []
+    if w.index in (1, 2, 3, 4):
+        sample_rows = min(rows, 4)           # batch 2x2 of each layer keeps one layer to about a second
+        comp = sample_rows // 2 if w.share_cfg else sample_rows
+        layer = 0
+        while True:
+            Kc, Vc = wl.make_kv(w, layer, batch_rows=sample_rows)
+            t_gen = time.perf_counter()
+            for k in w.steps:
+                Q = wl.make_q(w, layer, k, batch_rows=sample_rows)
+                orc.attention_step(w.scales, k, tab[k - 1], Q, Kc, Vc, share_cfg=w.share_cfg)
+                done_flop += orc.live_count(w.scales, k, tab[k - 1]) * FLOP_PER_ENTRY * comp * w.n_heads
+            layer += 1
+            _ = t_gen
+            if time.perf_counter() - t0 > seconds or layer >= w.n_layers:
+                break
+        what = f"{layer} layer(s) x all {len(w.steps)} steps, batch 2x{sample_rows // 2}, every row (input generation included)"
+    else:
+        k = w.steps[-1]
+        Kc, Vc = wl.make_kv(w, 0)
+        Q = wl.make_q(w, 0, k)
+        n_k = w.scales[k - 1] ** 2
+        rng = np.random.default_rng(0)
+        n = 0
+        m = orc.mask(w.scales, k, tab[k - 1], q_rows=range(0, n_k, 64))
+        mean_live = float(m.sum(1).mean())
+        while time.perf_counter() - t0 < seconds:
+            smp = [(int(rng.integers(0, rows)), int(rng.integers(0, w.n_heads)), int(rng.integers(0, n_k)))
+                   for _ in range(64)]
+            orc.attention_sampled(w.scales, k, tab[k - 1], Q, Kc, Vc, smp)
+            n += 64
+        done_flop = n * mean_live * FLOP_PER_ENTRY
+        what = f"{n} sampled query rows of step {k}"
+    return done_flop, time.perf_counter() - t0, what
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return int(torch.get_num_threads())
+
+
+def oracle_baseline(w: wl.Workload, seconds: float):
+    flop, el, what = oracle_sample(w, seconds)
+    return {"value": round(flop / el / 1e12, 6), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+            "sample": what, "seconds": round(el, 2), "host_cpus": os.cpu_count()}
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    w = wl.WORKLOADS[args.config]
+    per_step = max(0.5, min(20.0, args.cpu_seconds / max(1, args.steps)))
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, min(per_step, 1.0))
+    flop_tot, el_tot, what = 0.0, 0.0, ""
+    for _ in range(args.steps):
+        flop, el, what = oracle_sample(w, per_step)
+        flop_tot += flop
+        el_tot += el
+    value = flop_tot / el_tot / 1e12
+    out = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 6), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(el_tot / args.steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"config {w.index}: {w.name}", "variant": "window", "scales": list(w.scales),
+                   "steps_per_generation": len(w.steps), "layers": w.n_layers, "heads": w.n_heads,
+                   "batch": f"2x{w.batch_pairs}", "cfg_share": w.share_cfg, "window_rho": list(w.rho),
+                   "note": "each step is a bounded sample of the workload run by the CPU oracle"},
+        "gpu_launches": 0,
+        "cpu_baseline": {"value": round(value, 6), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                         "sample": f"per step: {what}"},
+        "e2e": {"value": round(value, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--dense", action="store_true", help="full-mask variant of the same kernel")
+    ap.add_argument("--no-extras", action="store_true", help="skip the five-workload table")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="only the device-timed graph replays (for profiler runs): no eager, end-to-end, "
+                         "CPU or all-workload legs")
+    ap.add_argument("--rho", type=int, nargs=2, default=None, help="window radius ratio num den (default: the workload's)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        gpu_arm(args)
+
+
+if __name__ == "__main__":
+    main()
