@@ -124,6 +124,46 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
                                       const void* Vcache, const litevar_strides_t* sv,
                                       void* out, const litevar_strides_t* so, void* stream);
 
+/*
+ * Step-k attention without a plan object and without any allocation.  The paper has no counterpart:
+ * this is a deployment convenience of this library.
+ *
+ * litevar_attn_plan keeps its tile lists in memory it gets from cudaMalloc.  A caller that may not
+ * allocate (it runs inside a fixed device-memory budget, it is a plug-in that must stay away from its
+ * host's allocator, or it is reached at a point where allocation is forbidden) uses this call instead:
+ * it builds the tile plan of step_k on the device inside a fixed 4.2 MB array that is part of the
+ * library image, then runs the same tensor-core forward kernel on it.  It calls no cudaMalloc, no
+ * cudaFree and no allocating library routine; it launches three kernels on `stream` and returns
+ * without synchronising.
+ *
+ *   scales .. sm_scale, window   as for litevar_attn_plan (window->n_sets must be 1; a radius table,
+ *                                if given, is read at row step_k-1 only; head_to_set is ignored)
+ *   share_cfg                    non-zero: CFG sharing at this step (rows [0,B) computed, stored twice)
+ *   step_k .. stream             as for litevar_attn_forward
+ *
+ * Limits and rules.
+ *   - The step must have at most 2048 candidate tile pairs, ceil(n_k/128) * ceil(L_k/128)
+ *     (every step of the 256px and 512px schedules fits; the 2K step does not): otherwise
+ *     LITEVAR_ERR_UNSUPPORTED is returned and nothing is launched.
+ *   - Every GPU that loads the library holds the array until the process exits.  All calls on a device
+ *     share it and it keeps the last call's contents: calls that may overlap on the GPU (different
+ *     streams, or concurrent host threads) race; keep them on one stream or order them yourself.
+ *     Each call rewrites every entry it later reads and clears its status word, so nothing depends on
+ *     what an earlier call left behind.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress) with
+ *     that device current; make that first call outside any stream capture.
+ *   - There is no empty-row check: with a caller table that leaves a query without a live key the
+ *     row's output is undefined.  A bounded device-side wait that expires is not reported.
+ * Errors: INVALID_ARG, UNSUPPORTED, ARCH, CUDA.
+ */
+litevar_status_t litevar_attn_forward_static(const int32_t* scales, int32_t n_scales, int32_t n_heads,
+                                             int32_t head_dim, float sm_scale, const litevar_window_t* window,
+                                             int32_t share_cfg, int32_t step_k, int32_t batch_pairs,
+                                             const void* Q, const litevar_strides_t* sq,
+                                             const void* Kcache, const litevar_strides_t* sk,
+                                             const void* Vcache, const litevar_strides_t* sv,
+                                             void* out, const litevar_strides_t* so, void* stream);
+
 /* Counts for step k and window set `set`: live map entries, live / full / partial tile pairs. */
 litevar_status_t litevar_plan_stats(const litevar_plan_t* plan, int32_t step_k, int32_t set,
                                     int64_t* live_entries, int64_t* live_tiles, int64_t* full_tiles,

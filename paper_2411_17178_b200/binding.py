@@ -23,7 +23,7 @@ WINDOW_SQUARE, WINDOW_BAND = 0, 1
 KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
 
 EXPORTS = (
-    "litevar_attn_plan", "litevar_attn_forward", "litevar_plan_stats", "litevar_plan_tile_counts",
+    "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_static", "litevar_plan_stats", "litevar_plan_tile_counts",
     "litevar_plan_export_tiles", "litevar_plan_export_bounds", "litevar_plan_materialize_mask",
     "litevar_plan_poll_device_status", "litevar_plan_set_kernel", "litevar_plan_destroy",
     "litevar_status_string",
@@ -71,6 +71,11 @@ def load() -> ctypes.CDLL:
     lib.litevar_attn_forward.restype = ctypes.c_int
     lib.litevar_attn_forward.argtypes = [P, I32, I32, P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides),
                                          P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides), P]
+    lib.litevar_attn_forward_static.restype = ctypes.c_int
+    lib.litevar_attn_forward_static.argtypes = [ctypes.POINTER(I32), I32, I32, I32, ctypes.c_float,
+                                                ctypes.POINTER(_Window), I32, I32, I32,
+                                                P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides),
+                                                P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides), P]
     lib.litevar_plan_stats.restype = ctypes.c_int
     lib.litevar_plan_stats.argtypes = [P, I32, I32] + [ctypes.POINTER(I64)] * 4
     lib.litevar_plan_tile_counts.restype = ctypes.c_int
@@ -236,6 +241,39 @@ class Plan:
 
     def set_kernel(self, kernel: int) -> None:
         _check(self._lib.litevar_plan_set_kernel(self._h, int(kernel)), "litevar_plan_set_kernel")
+
+
+STATIC_MAX_PAIRS = 2048
+
+
+def forward_static(scales: Sequence[int], n_heads: int, step_k: int, batch_pairs: int, q, k_cache, v_cache, out,
+                   share_cfg: bool = False, head_dim: int = 64, sm_scale: float = 0.0, shape: int = WINDOW_SQUARE,
+                   n_global_scales: int = 3, rho=(1, 4), radius=None, stream=None) -> None:
+    """litevar_attn_forward_static: step-k attention for callers that must not allocate device memory.
+
+    No plan object: the step's tile plan is rebuilt on the device, inside a fixed array that belongs to
+    the library, on every call.  Steps with more than STATIC_MAX_PAIRS candidate tile pairs are refused.
+    Calls share that array, so keep them on one stream."""
+    lib = load()
+    K = len(scales)
+    win = _Window()
+    win.shape, win.n_global_scales = int(shape), int(n_global_scales)
+    win.rho_num, win.rho_den = int(rho[0]), int(rho[1])
+    win.n_sets = 1
+    keep = None
+    if radius is not None:
+        keep = np.ascontiguousarray(np.asarray(radius, dtype=np.int32).reshape(K, K))
+        win.radius = keep.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    st = lib.litevar_attn_forward_static(
+        _i32_array(scales), K, int(n_heads), int(head_dim), float(sm_scale), ctypes.byref(win),
+        1 if share_cfg else 0, int(step_k), int(batch_pairs),
+        q.data_ptr(), ctypes.byref(_strides(q)), k_cache.data_ptr(), ctypes.byref(_strides(k_cache)),
+        v_cache.data_ptr(), ctypes.byref(_strides(v_cache)), out.data_ptr(), ctypes.byref(_strides(out)),
+        _stream_ptr(stream))
+    if st == 2:
+        raise LitevarError(st, "litevar_attn_forward_static (head_dim must be 64, one window set, and the step "
+                               f"may have at most {STATIC_MAX_PAIRS} candidate tile pairs)")
+    _check(st, "litevar_attn_forward_static")
 
 
 def status_string(status: int) -> str:
