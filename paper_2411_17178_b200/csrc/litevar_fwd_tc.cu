@@ -1,13 +1,23 @@
 // Tensor-core forward kernel for sm_100a: TMA-staged bf16 tiles, tcgen05 MMAs with TMEM
 // accumulators, fp32 online softmax, element mask from the plan's bit blocks.
 //
-// One CTA handles one (query tile, head, batch row) and walks the live key tiles of its query
-// tile in plan order.  Warp roles:
-//   warp 0      TMA producer (one lane): Q once, then K and V of every live key tile into a ring
-//   warp 1      TMEM allocation; one lane issues S = Q K^T and O += P V
-//   warps 2..5  softmax: thread = query row (TMEM lane); mask, running max/sum, P -> TMEM (bf16),
-//               O rescale when the row max moves, final normalise + store (twice under CFG sharing)
-// TMEM columns: S fp32 [0,128), O fp32 [128,192), P bf16x2 [192,256).
+// One CTA handles two adjacent query tiles ("halves", 128 queries each) of one (head, batch row) and
+// walks the union of their live key-tile lists in plan order, so every K/V tile is staged once for
+// both halves.  384 threads in three warpgroups:
+//   warp 0       TMA producer (one lane): Q of both halves, then K and V of every listed key tile into
+//                two rings of kStages tiles
+//   warp 1       TMEM allocation; one lane issues S_h = Q_h K^T and O_h += P_h V for both halves
+//   warps 4..7   softmax of half 0, warps 8..11 softmax of half 1: thread = query row (TMEM lane).
+//                One pass per key tile over 32-key chunks: mask, exponentials against the row's
+//                reference max, P to TMEM as packed bf16, fp32 row sum of those rounded values (so the
+//                normaliser matches the weights of the PV product), and the tile max on the side.
+//                Chunks without a live key for the whole warp are skipped.  The reference max is fixed
+//                by the first tile and moves only when a later tile exceeds it by more than 2^8; the
+//                accumulator is then rescaled and that tile redone (every stored probability stays
+//                <= 256, and the final divide makes the result exact).
+// The issue order S_0(i), PV_0(i-1), S_1(i), PV_1(i-1) lets the tensor pipe work on one half while the
+// other half is in its softmax.
+// TMEM columns: S_0 [0,128) S_1 [128,256) O_0 [256,320) O_1 [320,384) P_0 [384,448) P_1 [448,512).
 //
 // Every wait is bounded: when a wait runs out the CTA raises the plan's status word, drains its
 // outstanding copies, frees its TMEM and returns.
@@ -23,24 +33,22 @@ namespace litevar {
 
 namespace {
 
-constexpr int kStages = 2;
-constexpr int kThreads = 192;
+constexpr int kStages = 4;
+constexpr int kThreads = 384;
 constexpr uint32_t kTileBytes = kBlockN * kHeadDim * 2;  // 16 KB: 128 rows of 128 B
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 128, kColP = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;  // + 128 / 64 / 64 per half
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr float kRescaleThreshold = 8.f;  // log2 units
+constexpr int kNoTile = 0x7fffffff;
 
 struct SharedStorage {
-  alignas(1024) uint8_t q[kTileBytes];
+  alignas(1024) uint8_t q[2][kTileBytes];
   alignas(1024) uint8_t k[kStages][kTileBytes];
   alignas(1024) uint8_t v[kStages][kTileBytes];
-  alignas(8) uint64_t bar_q;
-  uint64_t bar_k[kStages];
-  uint64_t bar_v[kStages];
-  uint64_t bar_free[kStages];
-  uint64_t bar_s;
-  uint64_t bar_p;
-  uint64_t bar_o;
+  alignas(8) uint64_t q_full;
+  uint64_t k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
+  uint64_t s_full[2], s_free[2], p_full[2], p_free[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -93,9 +101,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
 
 // Bounded wait.  Returns false when another role gave up or the time limit passed; the caller then
 // leaves its loop and falls through to the common teardown.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status) {
-  if (mbar_try(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                            int32_t* status) {
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try(bar, parity)) return true;
@@ -108,6 +115,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status) {
+  if (mbar_try(bar, parity)) return true;
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
@@ -141,7 +154,8 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -153,18 +167,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
       "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
@@ -172,37 +175,84 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&t);
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+// Walk of the union of two ascending key-tile lists (the two halves of the CTA).
+struct UnionWalk {
+  const Pair* pairs;
+  int i0, e0, i1, e1;
+  int kt0, kt1;  // heads of the two lists (kNoTile when exhausted)
+  __device__ __forceinline__ void init(const Pair* p, int b0, int end0, int b1, int end1) {
+    pairs = p;
+    i0 = b0; e0 = end0; i1 = b1; e1 = end1;
+    kt0 = i0 < e0 ? __ldg(&pairs[i0].key_tile) : kNoTile;
+    kt1 = i1 < e1 ? __ldg(&pairs[i1].key_tile) : kNoTile;
+  }
+  __device__ __forceinline__ bool has() const { return kt0 != kNoTile || kt1 != kNoTile; }
+  // Next key tile and which halves list it; heads are refilled at once so that the loads overlap
+  // the caller's waits.
+  __device__ __forceinline__ int next(bool& live0, bool& live1) {
+    const int kt = min(kt0, kt1);
+    live0 = kt0 == kt;
+    live1 = kt1 == kt;
+    if (live0) kt0 = ++i0 < e0 ? __ldg(&pairs[i0].key_tile) : kNoTile;
+    if (live1) kt1 = ++i1 < e1 ? __ldg(&pairs[i1].key_tile) : kNoTile;
+    return kt;
+  }
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-              const __grid_constant__ CUtensorMap tm_v, FwdParams p) {
+              const __grid_constant__ CUtensorMap tm_v, FwdParams p, int n_q_tiles) {
   extern __shared__ uint8_t smem_raw[];
   SharedStorage& sm = *reinterpret_cast<SharedStorage*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const SetDesc sd = p.sets[p.head_to_set ? p.head_to_set[h] : 0];
-  const int pair_begin = sd.row_ptr[qt];
-  const int n_tiles = sd.row_ptr[qt + 1] - pair_begin;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int qt0 = 2 * blockIdx.x, qt1 = qt0 + 1;
+  const bool has1 = qt1 < n_q_tiles;
   volatile int* abort_flag = &sm.abort_flag;
 
   if (threadIdx.x == 0) {
-    mbar_init(&sm.bar_q, 1);
+    mbar_init(&sm.q_full, 1);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.bar_k[s], 1);
-      mbar_init(&sm.bar_v[s], 1);
-      mbar_init(&sm.bar_free[s], 1);
+      mbar_init(&sm.k_full[s], 1);
+      mbar_init(&sm.k_free[s], 1);
+      mbar_init(&sm.v_full[s], 1);
+      mbar_init(&sm.v_free[s], 1);
     }
-    mbar_init(&sm.bar_s, 1);
-    mbar_init(&sm.bar_p, 128);
-    mbar_init(&sm.bar_o, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sm.s_full[i], 1);
+      mbar_init(&sm.s_free[i], 4);
+      mbar_init(&sm.p_full[i], 4);
+      mbar_init(&sm.p_free[i], 1);
+    }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -213,146 +263,273 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // plan lookups (independent of the set-up above)
+  const SetDesc sd = p.sets[p.head_to_set ? p.head_to_set[h] : 0];
+  const int beg0 = __ldg(&sd.row_ptr[qt0]), end0 = __ldg(&sd.row_ptr[qt0 + 1]);
+  const int beg1 = end0, end1 = has1 ? __ldg(&sd.row_ptr[qt1 + 1]) : end0;
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  if (warp == 0) {
-    if (lane == 0 && n_tiles > 0) {
+  if (warp < 4) {
+    if (warp == 0 && lane == 0 && end1 > beg0) {
       // ---------------------------------------------------------------- TMA producer
-      mbar_expect_tx(&sm.bar_q, kTileBytes);
-      tma_load_4d(sm.q, &tm_q, 0, qt * kBlockM, h, b, &sm.bar_q);
+      const bool ld0 = end0 > beg0, ld1 = end1 > beg1;
+      mbar_expect_tx(&sm.q_full, (ld0 ? kTileBytes : 0u) + (ld1 ? kTileBytes : 0u));
+      if (ld0) tma_load_4d(sm.q[0], &tm_q, 0, qt0 * kBlockM, h, b, &sm.q_full);
+      if (ld1) tma_load_4d(sm.q[1], &tm_q, 0, qt1 * kBlockM, h, b, &sm.q_full);
+      UnionWalk w;
+      w.init(sd.pairs, beg0, end0, beg1, end1);
       int issued = 0;
-      for (int i = 0; i < n_tiles; ++i) {
+      for (int i = 0; w.has(); ++i) {
+        bool l0, l1;
+        const int t0 = w.next(l0, l1) * kBlockN;
         const int s = i % kStages, n = i / kStages;
-        if (n > 0 && !mbar_wait(&sm.bar_free[s], (uint32_t)((n - 1) & 1), abort_flag, p.status)) break;
-        const int t0 = sd.pairs[pair_begin + i].key_tile * kBlockN;
-        mbar_expect_tx(&sm.bar_k[s], kTileBytes);
-        tma_load_4d(sm.k[s], &tm_k, 0, t0, h, b, &sm.bar_k[s]);
-        mbar_expect_tx(&sm.bar_v[s], kTileBytes);
-        tma_load_4d(sm.v[s], &tm_v, 0, t0, h, b, &sm.bar_v[s]);
+        if (n > 0 && !mbar_wait(&sm.k_free[s], (uint32_t)((n - 1) & 1), abort_flag, p.status)) break;
+        mbar_expect_tx(&sm.k_full[s], kTileBytes);
+        tma_load_4d(sm.k[s], &tm_k, 0, t0, h, b, &sm.k_full[s]);
+        if (n > 0 && !mbar_wait(&sm.v_free[s], (uint32_t)((n - 1) & 1), abort_flag, p.status)) {
+          // the K copy just issued is still in flight
+          const unsigned long long ts = global_ns();
+          while (!mbar_try(&sm.k_full[s], (uint32_t)(n & 1)))
+            if (global_ns() - ts > kWaitLimitNs) break;
+          break;
+        }
+        mbar_expect_tx(&sm.v_full[s], kTileBytes);
+        tma_load_4d(sm.v[s], &tm_v, 0, t0, h, b, &sm.v_full[s]);
         issued = i + 1;
       }
       if (*abort_flag) {
         // wait (bounded) for copies still in flight before the CTA may exit
-        (void)mbar_wait(&sm.bar_q, 0u, abort_flag, p.status);
+        const unsigned long long ts = global_ns();
+        while (!mbar_try(&sm.q_full, 0u))
+          if (global_ns() - ts > kWaitLimitNs) break;
         for (int i = issued > kStages ? issued - kStages : 0; i < issued; ++i) {
           const int s = i % kStages, n = i / kStages;
-          const unsigned long long t0 = global_ns();
-          while (!(mbar_try(&sm.bar_k[s], (uint32_t)(n & 1)) && mbar_try(&sm.bar_v[s], (uint32_t)(n & 1))))
-            if (global_ns() - t0 > kWaitLimitNs) break;
+          while (!(mbar_try(&sm.k_full[s], (uint32_t)(n & 1)) && mbar_try(&sm.v_full[s], (uint32_t)(n & 1))))
+            if (global_ns() - ts > 2 * kWaitLimitNs) break;
         }
       }
-    }
-  } else if (warp == 1) {
-    if (lane == 0 && n_tiles > 0) {
+    } else if (warp == 1 && lane == 0 && end1 > beg0) {
       // ---------------------------------------------------------------- MMA issuer
-      const uint64_t q_desc = make_desc(smem_u32(sm.q));
-      bool ok = mbar_wait(&sm.bar_q, 0u, abort_flag, p.status);
-      for (int i = 0; ok && i < n_tiles; ++i) {
+      const uint64_t q_desc[2] = {make_desc(smem_u32(sm.q[0])), make_desc(smem_u32(sm.q[1]))};
+      UnionWalk w;
+      w.init(sd.pairs, beg0, end0, beg1, end1);
+      bool ok = mbar_wait(&sm.q_full, 0u, abort_flag, p.status);
+      int n_s[2] = {0, 0}, n_pv[2] = {0, 0};
+      bool prev_live[2] = {false, false};
+      int prev_stage = 0;
+      uint32_t prev_phase = 0;
+      for (int i = 0; ok; ++i) {
+        const bool have = w.has();
+        bool live[2] = {false, false};
         const int s = i % kStages;
         const uint32_t ph = (uint32_t)((i / kStages) & 1);
-        if (!(ok = mbar_wait(&sm.bar_k[s], ph, abort_flag, p.status))) break;
-        tc_fence_after();
-        const uint64_t k_desc = make_desc(smem_u32(sm.k[s]));
+        uint64_t k_desc = 0;
+        if (have) {
+          (void)w.next(live[0], live[1]);
+          if (!(ok = mbar_wait(&sm.k_full[s], ph, abort_flag, p.status))) break;
+          tc_fence_after();
+          k_desc = make_desc(smem_u32(sm.k[s]));
+        }
+        bool v_ready = false;
+        const uint64_t v_desc = make_desc(smem_u32(sm.v[prev_stage]));
 #pragma unroll
-        for (int kk = 0; kk < kHeadDim / 16; ++kk)  // 16 bf16 = 32 B per step inside the swizzle row
-          mma_ss(tmem + kColS, q_desc + 2 * kk, k_desc + 2 * kk, kIdescQK, kk > 0 ? 1u : 0u);
-        mma_commit(&sm.bar_s);
-        if (!(ok = mbar_wait(&sm.bar_p, (uint32_t)(i & 1), abort_flag, p.status))) break;
-        if (!(ok = mbar_wait(&sm.bar_v[s], ph, abort_flag, p.status))) break;
-        tc_fence_after();
-        const uint64_t v_desc = make_desc(smem_u32(sm.v[s]));
+        for (int hh = 0; hh < 2; ++hh) {
+          if (have && live[hh]) {
+            if (n_s[hh] > 0) {  // the softmax group has copied the previous S_hh into registers
+              if (!(ok = mbar_wait(&sm.s_free[hh], (uint32_t)((n_s[hh] - 1) & 1), abort_flag, p.status))) break;
+              tc_fence_after();
+            }
 #pragma unroll
-        for (int kk = 0; kk < kBlockN / 16; ++kk)  // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns
-          mma_ts(tmem + kColO, tmem + kColP + 8 * kk, v_desc + (uint64_t)(2048 >> 4) * kk, kIdescPV,
-                 (i > 0 || kk > 0) ? 1u : 0u);
-        mma_commit(&sm.bar_free[s]);
-        if (i == n_tiles - 1) mma_commit(&sm.bar_o);
+            for (int kk = 0; kk < kHeadDim / 16; ++kk)  // 16 bf16 = 32 B per step inside the swizzle row
+              mma_ss(tmem + kColS + 128 * hh, q_desc[hh] + 2 * kk, k_desc + 2 * kk, kIdescQK, kk > 0 ? 1u : 0u);
+            mma_commit(&sm.s_full[hh]);
+            ++n_s[hh];
+          }
+          if (i > 0 && prev_live[hh]) {
+            if (!(ok = mbar_wait(&sm.p_full[hh], (uint32_t)(n_pv[hh] & 1), abort_flag, p.status))) break;
+            if (!v_ready) {
+              if (!(ok = mbar_wait(&sm.v_full[prev_stage], prev_phase, abort_flag, p.status))) break;
+              v_ready = true;
+            }
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < kBlockN / 16; ++kk)  // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns
+              mma_ts(tmem + kColO + 64 * hh, tmem + kColP + 64 * hh + 8 * kk, v_desc + (uint64_t)(2048 >> 4) * kk,
+                     kIdescPV, (n_pv[hh] > 0 || kk > 0) ? 1u : 0u);
+            mma_commit(&sm.p_free[hh]);
+            ++n_pv[hh];
+          }
+        }
+        if (!ok) break;
+        if (have) mma_commit(&sm.k_free[s]);
+        if (i > 0) mma_commit(&sm.v_free[prev_stage]);
+        if (!have) break;
+        prev_live[0] = live[0];
+        prev_live[1] = live[1];
+        prev_stage = s;
+        prev_phase = ph;
       }
     }
-  } else if (n_tiles > 0) {
-    // ------------------------------------------------------------------ softmax + epilogue
-    const int lane_group = warp & 3;  // TMEM lanes this warp may touch: 32*lane_group .. +31
-    const int m = lane_group * 32 + lane;
-    const int q = qt * kBlockM + m;
-    const uint32_t tbase = tmem + ((uint32_t)(lane_group * 32) << 16);
-    const float sc = p.sm_scale * 1.4426950408889634f;
-    float row_max = -INFINITY, row_sum = 0.f;
-    bool ok = true;
-    uint32_t r[32];
-    for (int i = 0; i < n_tiles; ++i) {
-      const Pair pr = sd.pairs[pair_begin + i];
-      uint4 bits4 = make_uint4(~0u, ~0u, ~0u, ~0u);
-      if (pr.mask_block >= 0) bits4 = sd.mask[(size_t)pr.mask_block * kBlockM + m];
-      const uint32_t bits[4] = {bits4.x, bits4.y, bits4.z, bits4.w};
-      if (!(ok = mbar_wait(&sm.bar_s, (uint32_t)(i & 1), abort_flag, p.status))) break;
-      tc_fence_after();
-      // pass 1: row maximum over live keys
-      float mx = -INFINITY;
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue of one half
+    const int hh = (warp - 4) >> 2;
+    const int qt = hh ? qt1 : qt0;
+    const int pbeg = hh ? beg1 : beg0;
+    const int n_tiles = (hh ? end1 : end0) - pbeg;
+    if (n_tiles > 0) {
+      const int lane_group = warp & 3;  // TMEM lanes this warp may touch: 32*lane_group .. +31
+      const int m = lane_group * 32 + lane;
+      const int q = qt * kBlockM + m;
+      const uint32_t tlane = tmem + ((uint32_t)(lane_group * 32) << 16);
+      const uint32_t tS = tlane + kColS + 128 * hh, tO = tlane + kColO + 64 * hh, tP = tlane + kColP + 64 * hh;
+      const float sc = p.sm_scale * 1.4426950408889634f;
+      float row_max = -INFINITY, row_sum = 0.f;  // row_max: the score the stored probabilities refer to
+      bool ok = true;
+      Pair pr = sd.pairs[pbeg];
+      uint4 mk = make_uint4(~0u, ~0u, ~0u, ~0u);
+      if (pr.mask_block >= 0) mk = __ldg(&sd.mask[(size_t)pr.mask_block * kBlockM + m]);
+      for (int j = 0; j < n_tiles; ++j) {
+        // next pair's mask words travel while this tile is processed
+        Pair pr_next = pr;
+        uint4 mk_next = make_uint4(~0u, ~0u, ~0u, ~0u);
+        if (j + 1 < n_tiles) {
+          pr_next = sd.pairs[pbeg + j + 1];
+          if (pr_next.mask_block >= 0) mk_next = __ldg(&sd.mask[(size_t)pr_next.mask_block * kBlockM + m]);
+        }
+        const bool partial = pr.mask_block >= 0;
+        const uint32_t wbits[4] = {mk.x, mk.y, mk.z, mk.w};
+        // per 32-key chunk, uniform over the warp: 0 = no live key (skipped), 1 = mixed, 2 = all live
+        int chunk_kind[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld32(tbase + kColS + 32 * c, r);
-        tmem_wait_ld();
+        for (int c = 0; c < 4; ++c) {
+          chunk_kind[c] = 2;
+          if (partial)
+            chunk_kind[c] = !__any_sync(0xffffffffu, wbits[c] != 0u) ? 0
+                            : (__all_sync(0xffffffffu, wbits[c] == 0xffffffffu) ? 2 : 1);
+        }
+        if (!(ok = mbar_wait(&sm.s_full[hh], (uint32_t)(j & 1), abort_flag, p.status))) break;
+        tc_fence_after();
+        uint32_t r[32];
+        float tile_max = -INFINITY;
+        if (j == 0) {
+          // the first tile fixes the reference max before any probability is formed
+          float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-        for (int e = 0; e < 32; ++e)
-          if ((bits[c] >> e) & 1u) mx = fmaxf(mx, __uint_as_float(r[e]));
+          for (int c = 0; c < 4; ++c) {
+            if (chunk_kind[c] == 0) continue;
+            tmem_ld32(tS + 32 * c, r);
+            tmem_wait_ld();
+            if (chunk_kind[c] == 1) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (!((wbits[c] >> e) & 1u)) r[e] = 0xff800000u;  // -inf
+            }
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+              mx0 = max3(mx0, __uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
+              mx1 = max3(mx1, __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+            }
+          }
+          row_max = fmaxf(mx0, mx1);
+        } else {
+          // PV of the previous tile done: P_hh may be rewritten, O_hh is stable
+          if (!(ok = mbar_wait(&sm.p_free[hh], (uint32_t)((j - 1) & 1), abort_flag, p.status))) break;
+          tc_fence_after();
+        }
+        float psum = 0.f;
+        for (int attempt = 0;; ++attempt) {
+          // probabilities against row_max, P as packed bf16 into TMEM, the fp32 sum of P, and the tile max
+          const float msc = row_max == -INFINITY ? 0.f : row_max * sc;
+          float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t pk[16];
+            if (chunk_kind[c] != 0) {
+              tmem_ld32(tS + 32 * c, r);
+              tmem_wait_ld();
+              if (chunk_kind[c] == 1) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                  if (!((wbits[c] >> e) & 1u)) r[e] = 0xff800000u;  // -inf
+              }
+#pragma unroll
+              for (int e = 0; e < 32; e += 4) {
+                mx0 = max3(mx0, __uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
+                mx1 = max3(mx1, __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                const float p0 = fast_exp2(fmaf(__uint_as_float(r[e + 0]), sc, -msc));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), sc, -msc));
+                const float p2 = fast_exp2(fmaf(__uint_as_float(r[e + 2]), sc, -msc));
+                const float p3 = fast_exp2(fmaf(__uint_as_float(r[e + 3]), sc, -msc));
+                const uint32_t k0 = pack_bf16(p0, p1), k1 = pack_bf16(p2, p3);
+                pk[(e >> 1) + 0] = k0;
+                pk[(e >> 1) + 1] = k1;
+                // the row sum takes the rounded probabilities, the very weights the PV product uses
+                ps0 += __uint_as_float(k0 << 16);
+                ps1 += __uint_as_float(k0 & 0xffff0000u);
+                ps2 += __uint_as_float(k1 << 16);
+                ps3 += __uint_as_float(k1 & 0xffff0000u);
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) pk[e] = 0u;
+            }
+            tmem_st16(tP + 16 * c, pk);
+          }
+          psum = (ps0 + ps1) + (ps2 + ps3);
+          tile_max = fmaxf(mx0, mx1);
+          // the reference max moves only when the tile exceeds it by more than the threshold; then the
+          // accumulator and the sum are rescaled and the tile is redone (rare after the first tiles)
+          const bool exceed = (tile_max - row_max) * sc > kRescaleThreshold;  // false for tile_max = -inf
+          if (attempt > 0 || !__any_sync(0xffffffffu, exceed)) break;
+          const float alpha = (exceed && row_max != -INFINITY) ? fast_exp2((row_max - tile_max) * sc) : 1.f;
+          if (exceed) row_max = tile_max;
+          row_sum *= alpha;
+          uint32_t o[16];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld16(tO + 16 * c, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st16(tO + 16 * c, o);
+          }
+        }
+        row_sum += psum;
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&sm.s_free[hh]);  // S_hh may be overwritten by the next key tile
+          mbar_arrive(&sm.p_full[hh]);
+        }
+        pr = pr_next;
+        mk = mk_next;
       }
-      const float new_max = fmaxf(row_max, mx);
-      const float alpha = row_max == -INFINITY ? 1.f : exp2f((row_max - new_max) * sc);
-      const float msc = new_max == -INFINITY ? 0.f : new_max * sc;
-      if (i > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+      if (ok && (ok = mbar_wait(&sm.p_free[hh], (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status))) {
+        tc_fence_after();
+        const float inv = 1.f / row_sum;
+        uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st;
+        uint16_t* orow2 = orow + (int64_t)p.share_offset * p.o_sb;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          tmem_ld32(tbase + kColO + 32 * c, r);
+          uint32_t r[32];
+          tmem_ld32(tO + 32 * c, r);
           tmem_wait_ld();
+          if (q < p.n_k) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-          tmem_st32(tbase + kColO + 32 * c, r);
-        }
-      }
-      // pass 2: probabilities, row sum (from unrounded p), P as packed bf16 into TMEM
-      float psum = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld32(tbase + kColS + 32 * c, r);
-        tmem_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float p0 = ((bits[c] >> e) & 1u) ? exp2f(fmaf(__uint_as_float(r[e]), sc, -msc)) : 0.f;
-          float p1 = ((bits[c] >> (e + 1)) & 1u) ? exp2f(fmaf(__uint_as_float(r[e + 1]), sc, -msc)) : 0.f;
-          psum += p0 + p1;
-          pk[e >> 1] = pack_bf16(p0, p1);
-        }
-        tmem_st16(tbase + kColP + 16 * c, pk);
-      }
-      row_sum = row_sum * alpha + psum;
-      row_max = new_max;
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&sm.bar_p);
-    }
-    if (ok && (ok = mbar_wait(&sm.bar_o, 0u, abort_flag, p.status))) {
-      tc_fence_after();
-      const float inv = 1.f / row_sum;
-      uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st;
-      uint16_t* orow2 = orow + (int64_t)p.share_offset * p.o_sb;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        tmem_ld32(tbase + kColO + 32 * c, r);
-        tmem_wait_ld();
-        if (q < p.n_k) {
-#pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 o4;
-            o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
-            o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-            o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-            o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + 32 * c + e) = o4;
-            if (p.share_offset > 0) *reinterpret_cast<uint4*>(orow2 + 32 * c + e) = o4;
+            for (int e = 0; e < 32; e += 8) {
+              uint4 o4;
+              o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
+              o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+              o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+              o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+              *reinterpret_cast<uint4*>(orow + 32 * c + e) = o4;
+              if (p.share_offset > 0) *reinterpret_cast<uint4*>(orow2 + 32 * c + e) = o4;
+            }
           }
         }
       }
@@ -422,8 +599,8 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
       !encode_map(&tm_k, p.k, p.L_k, p.n_heads, p.batch_computed, p.k_st, p.k_sh, p.k_sb) ||
       !encode_map(&tm_v, p.v, p.L_k, p.n_heads, p.batch_computed, p.v_st, p.v_sh, p.v_sb))
     return LITEVAR_ERR_INVALID_ARG;
-  dim3 grid((unsigned)n_q_tiles, (unsigned)p.n_heads, (unsigned)p.batch_computed);
-  fwd_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+  dim3 grid((unsigned)((n_q_tiles + 1) / 2), (unsigned)p.n_heads, (unsigned)p.batch_computed);
+  fwd_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p, n_q_tiles);
   if (cudaGetLastError() != cudaSuccess) return LITEVAR_ERR_CUDA;
   return LITEVAR_OK;
 }
