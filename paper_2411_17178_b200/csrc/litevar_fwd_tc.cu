@@ -6,18 +6,19 @@
 // both halves.  384 threads in three warpgroups:
 //   warp 0       TMA producer (one lane): Q of both halves, then K and V of every listed key tile into
 //                two rings of kStages tiles
-//   warp 1       TMEM allocation; one lane issues S_h = Q_h K^T and O_h += P_h V for both halves
+//   warp 1       TMEM allocation; one lane issues, per half h, O_h += P_h V (previous tile) and then
+//                S_h = Q_h K^T (next tile); the two halves alternate, so the tensor pipe works for one
+//                half while the other is in its softmax
 //   warps 4..7   softmax of half 0, warps 8..11 softmax of half 1: thread = query row (TMEM lane).
-//                One pass per key tile over 32-key chunks: mask, exponentials against the row's
-//                reference max, P to TMEM as packed bf16, fp32 row sum of those rounded values (so the
-//                normaliser matches the weights of the PV product), and the tile max on the side.
-//                Chunks without a live key for the whole warp are skipped.  The reference max is fixed
-//                by the first tile and moves only when a later tile exceeds it by more than 2^8; the
-//                accumulator is then rescaled and that tile redone (every stored probability stays
-//                <= 256, and the final divide makes the result exact).
-// The issue order S_0(i), PV_0(i-1), S_1(i), PV_1(i-1) lets the tensor pipe work on one half while the
-// other half is in its softmax.
-// TMEM columns: S_0 [0,128) S_1 [128,256) O_0 [256,320) O_1 [320,384) P_0 [384,448) P_1 [448,512).
+//                Pass 1 over 32-key chunks: element mask (mixed chunks only, written back to TMEM) and
+//                the exact row max of the tile.  The row's reference max moves only when the tile
+//                exceeds it by more than 2^8; only then is the accumulator rescaled.  Pass 2:
+//                exponentials against the reference, P as packed bf16 written over the first half of
+//                S_h's own columns.  Chunks without a live key for the whole warp are skipped.
+// Row sums come from the tensor pipe: the B operand of the PV product is V (64 columns) followed by a
+// block of ones (16 columns), so accumulator column 64 holds sum_t P[q,t] of the very bf16 weights the
+// output uses; no per-element add is issued.
+// TMEM columns: S_0/P_0 [0,128)  S_1/P_1 [128,256)  O_0 [256,336)  O_1 [336,416).
 //
 // Every wait is bounded: when a wait runs out the CTA raises the plan's status word, drains its
 // outstanding copies, frees its TMEM and returns.
@@ -37,7 +38,8 @@ constexpr int kStages = 4;
 constexpr int kThreads = 384;
 constexpr uint32_t kTileBytes = kBlockN * kHeadDim * 2;  // 16 KB: 128 rows of 128 B
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;  // + 128 / 64 / 64 per half
+constexpr uint32_t kColS = 0, kColO = 256;  // + 128 / kOutCols per half; P_h overlays S_h
+constexpr int kOutCols = kHeadDim + 16;      // V columns + the ones block (row sums)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr int kNoTile = 0x7fffffff;
@@ -46,9 +48,10 @@ struct SharedStorage {
   alignas(1024) uint8_t q[2][kTileBytes];
   alignas(1024) uint8_t k[kStages][kTileBytes];
   alignas(1024) uint8_t v[kStages][kTileBytes];
+  alignas(1024) uint8_t ones[kTileBytes];  // bf16 1.0 everywhere: second N block of the PV product's B operand
   alignas(8) uint64_t q_full;
   uint64_t k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
-  uint64_t s_full[2], s_free[2], p_full[2], p_free[2];
+  uint64_t s_full[2], p_full[2], o_full[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -59,7 +62,7 @@ struct SharedStorage {
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) |
                               ((uint32_t)(kBlockM >> 4) << 24);
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) |
-                              ((uint32_t)(kHeadDim >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
+                              ((uint32_t)(kOutCols >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -70,6 +73,12 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
   return (uint64_t)((saddr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
          (2ull << 61);
+}
+// MN-major operand wider than one 64-element block: the leading-dimension byte offset (bits 16-29)
+// is the distance from the first block of N columns to the next one.
+__device__ __forceinline__ uint64_t make_desc_mn(uint32_t saddr, uint32_t next_block_bytes) {
+  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((next_block_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -167,6 +176,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -249,9 +269,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.s_free[i], 4);
       mbar_init(&sm.p_full[i], 4);
-      mbar_init(&sm.p_free[i], 1);
+      mbar_init(&sm.o_full[i], 1);
     }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -262,6 +281,12 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  {  // the ones block; made visible to the tensor pipe (async proxy) before the barrier below
+    uint4* o4 = reinterpret_cast<uint4*>(sm.ones);
+    for (int i = threadIdx.x; i < (int)(kTileBytes / 16); i += kThreads)
+      o4[i] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   // plan lookups (independent of the set-up above)
   const SetDesc sd = p.sets[p.head_to_set ? p.head_to_set[h] : 0];
@@ -317,7 +342,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       UnionWalk w;
       w.init(sd.pairs, beg0, end0, beg1, end1);
       bool ok = mbar_wait(&sm.q_full, 0u, abort_flag, p.status);
-      int n_s[2] = {0, 0}, n_pv[2] = {0, 0};
+      int n_pv[2] = {0, 0};
       bool prev_live[2] = {false, false};
       int prev_stage = 0;
       uint32_t prev_phase = 0;
@@ -334,21 +359,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
           k_desc = make_desc(smem_u32(sm.k[s]));
         }
         bool v_ready = false;
-        const uint64_t v_desc = make_desc(smem_u32(sm.v[prev_stage]));
+        const uint32_t v_addr = smem_u32(sm.v[prev_stage]);
+        const uint64_t v_desc = make_desc_mn(v_addr, smem_u32(sm.ones) - v_addr);
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
-          if (have && live[hh]) {
-            if (n_s[hh] > 0) {  // the softmax group has copied the previous S_hh into registers
-              if (!(ok = mbar_wait(&sm.s_free[hh], (uint32_t)((n_s[hh] - 1) & 1), abort_flag, p.status))) break;
-              tc_fence_after();
-            }
-#pragma unroll
-            for (int kk = 0; kk < kHeadDim / 16; ++kk)  // 16 bf16 = 32 B per step inside the swizzle row
-              mma_ss(tmem + kColS + 128 * hh, q_desc[hh] + 2 * kk, k_desc + 2 * kk, kIdescQK, kk > 0 ? 1u : 0u);
-            mma_commit(&sm.s_full[hh]);
-            ++n_s[hh];
-          }
-          if (i > 0 && prev_live[hh]) {
+          if (i > 0 && prev_live[hh]) {  // O_hh += P_hh [V | 1]; P_hh sits in S_hh's columns
             if (!(ok = mbar_wait(&sm.p_full[hh], (uint32_t)(n_pv[hh] & 1), abort_flag, p.status))) break;
             if (!v_ready) {
               if (!(ok = mbar_wait(&sm.v_full[prev_stage], prev_phase, abort_flag, p.status))) break;
@@ -357,10 +372,16 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < kBlockN / 16; ++kk)  // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns
-              mma_ts(tmem + kColO + 64 * hh, tmem + kColP + 64 * hh + 8 * kk, v_desc + (uint64_t)(2048 >> 4) * kk,
-                     kIdescPV, (n_pv[hh] > 0 || kk > 0) ? 1u : 0u);
-            mma_commit(&sm.p_free[hh]);
+              mma_ts(tmem + kColO + kOutCols * hh, tmem + kColS + 128 * hh + 8 * kk,
+                     v_desc + (uint64_t)(2048 >> 4) * kk, kIdescPV, (n_pv[hh] > 0 || kk > 0) ? 1u : 0u);
+            mma_commit(&sm.o_full[hh]);
             ++n_pv[hh];
+          }
+          if (have && live[hh]) {  // S_hh = Q_hh K^T, after the PV above in issue order
+#pragma unroll
+            for (int kk = 0; kk < kHeadDim / 16; ++kk)  // 16 bf16 = 32 B per step inside the swizzle row
+              mma_ss(tmem + kColS + 128 * hh, q_desc[hh] + 2 * kk, k_desc + 2 * kk, kIdescQK, kk > 0 ? 1u : 0u);
+            mma_commit(&sm.s_full[hh]);
           }
         }
         if (!ok) break;
@@ -384,9 +405,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       const int m = lane_group * 32 + lane;
       const int q = qt * kBlockM + m;
       const uint32_t tlane = tmem + ((uint32_t)(lane_group * 32) << 16);
-      const uint32_t tS = tlane + kColS + 128 * hh, tO = tlane + kColO + 64 * hh, tP = tlane + kColP + 64 * hh;
+      const uint32_t tS = tlane + kColS + 128 * hh, tO = tlane + kColO + kOutCols * hh;
       const float sc = p.sm_scale * 1.4426950408889634f;
-      float row_max = -INFINITY, row_sum = 0.f;  // row_max: the score the stored probabilities refer to
+      float row_max = -INFINITY;  // the score the stored probabilities refer to
       bool ok = true;
       Pair pr = sd.pairs[pbeg];
       uint4 mk = make_uint4(~0u, ~0u, ~0u, ~0u);
@@ -403,94 +424,51 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const uint32_t wbits[4] = {mk.x, mk.y, mk.z, mk.w};
         // per 32-key chunk, uniform over the warp: 0 = no live key (skipped), 1 = mixed, 2 = all live
         int chunk_kind[4];
+        bool any_mixed = false;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           chunk_kind[c] = 2;
           if (partial)
             chunk_kind[c] = !__any_sync(0xffffffffu, wbits[c] != 0u) ? 0
                             : (__all_sync(0xffffffffu, wbits[c] == 0xffffffffu) ? 2 : 1);
+          any_mixed |= chunk_kind[c] == 1;
         }
+        // S_hh(j) complete; in issue order this also means the PV product of tile j-1 is complete
         if (!(ok = mbar_wait(&sm.s_full[hh], (uint32_t)(j & 1), abort_flag, p.status))) break;
         tc_fence_after();
-        uint32_t r[32];
-        float tile_max = -INFINITY;
-        if (j == 0) {
-          // the first tile fixes the reference max before any probability is formed
-          float mx0 = -INFINITY, mx1 = -INFINITY;
+        uint32_t r[2][32];
+        // ---- pass 1: mask the mixed chunks (written back) and take the row max of the tile
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+        tmem_ld32(tS, r[0]);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            if (chunk_kind[c] == 0) continue;
-            tmem_ld32(tS + 32 * c, r);
-            tmem_wait_ld();
-            if (chunk_kind[c] == 1) {
+        for (int c = 0; c < 4; ++c) {
+          uint32_t* rc = r[c & 1];
+          tmem_wait_ld();
+          if (c + 1 < 4) tmem_ld32(tS + 32 * (c + 1), r[(c + 1) & 1]);
+          if (chunk_kind[c] == 0) continue;
+          if (chunk_kind[c] == 1) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (!((wbits[c] >> e) & 1u)) r[e] = 0xff800000u;  // -inf
-            }
-#pragma unroll
-            for (int e = 0; e < 32; e += 4) {
-              mx0 = max3(mx0, __uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
-              mx1 = max3(mx1, __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-            }
+            for (int e = 0; e < 32; ++e)
+              if (!((wbits[c] >> e) & 1u)) rc[e] = 0xff800000u;  // -inf
+            tmem_st32(tS + 32 * c, rc);
           }
-          row_max = fmaxf(mx0, mx1);
-        } else {
-          // PV of the previous tile done: P_hh may be rewritten, O_hh is stable
-          if (!(ok = mbar_wait(&sm.p_free[hh], (uint32_t)((j - 1) & 1), abort_flag, p.status))) break;
-          tc_fence_after();
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            mx0 = max3(mx0, __uint_as_float(rc[e + 0]), __uint_as_float(rc[e + 1]));
+            mx1 = max3(mx1, __uint_as_float(rc[e + 2]), __uint_as_float(rc[e + 3]));
+          }
         }
-        float psum = 0.f;
-        for (int attempt = 0;; ++attempt) {
-          // probabilities against row_max, P as packed bf16 into TMEM, the fp32 sum of P, and the tile max
-          const float msc = row_max == -INFINITY ? 0.f : row_max * sc;
-          float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
-          float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t pk[16];
-            if (chunk_kind[c] != 0) {
-              tmem_ld32(tS + 32 * c, r);
-              tmem_wait_ld();
-              if (chunk_kind[c] == 1) {
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                  if (!((wbits[c] >> e) & 1u)) r[e] = 0xff800000u;  // -inf
-              }
-#pragma unroll
-              for (int e = 0; e < 32; e += 4) {
-                mx0 = max3(mx0, __uint_as_float(r[e + 0]), __uint_as_float(r[e + 1]));
-                mx1 = max3(mx1, __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                const float p0 = fast_exp2(fmaf(__uint_as_float(r[e + 0]), sc, -msc));
-                const float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), sc, -msc));
-                const float p2 = fast_exp2(fmaf(__uint_as_float(r[e + 2]), sc, -msc));
-                const float p3 = fast_exp2(fmaf(__uint_as_float(r[e + 3]), sc, -msc));
-                const uint32_t k0 = pack_bf16(p0, p1), k1 = pack_bf16(p2, p3);
-                pk[(e >> 1) + 0] = k0;
-                pk[(e >> 1) + 1] = k1;
-                // the row sum takes the rounded probabilities, the very weights the PV product uses
-                ps0 += __uint_as_float(k0 << 16);
-                ps1 += __uint_as_float(k0 & 0xffff0000u);
-                ps2 += __uint_as_float(k1 << 16);
-                ps3 += __uint_as_float(k1 & 0xffff0000u);
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 16; ++e) pk[e] = 0u;
-            }
-            tmem_st16(tP + 16 * c, pk);
-          }
-          psum = (ps0 + ps1) + (ps2 + ps3);
-          tile_max = fmaxf(mx0, mx1);
-          // the reference max moves only when the tile exceeds it by more than the threshold; then the
-          // accumulator and the sum are rescaled and the tile is redone (rare after the first tiles)
-          const bool exceed = (tile_max - row_max) * sc > kRescaleThreshold;  // false for tile_max = -inf
-          if (attempt > 0 || !__any_sync(0xffffffffu, exceed)) break;
-          const float alpha = (exceed && row_max != -INFINITY) ? fast_exp2((row_max - tile_max) * sc) : 1.f;
-          if (exceed) row_max = tile_max;
-          row_sum *= alpha;
+        const float tile_max = fmaxf(mx0, mx1);
+        // the reference max moves only when the tile exceeds it by more than the threshold
+        float alpha = 1.f;
+        if ((tile_max - row_max) * sc > kRescaleThreshold) {  // false for tile_max = -inf, true for row_max = -inf
+          if (row_max != -INFINITY) alpha = fast_exp2((row_max - tile_max) * sc);
+          row_max = tile_max;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // accumulator and row sum follow the reference
           uint32_t o[16];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < kOutCols / 16; ++c) {
             tmem_ld16(tO + 16 * c, o);
             tmem_wait_ld();
 #pragma unroll
@@ -498,22 +476,45 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             tmem_st16(tO + 16 * c, o);
           }
         }
-        row_sum += psum;
+        if (any_mixed) tmem_wait_st();  // the masked scores are read back below
+        // ---- pass 2: probabilities against the reference; P (packed bf16) over S_hh's first 64 columns
+        const float msc = row_max == -INFINITY ? 0.f : row_max * sc;
+        tmem_ld32(tS, r[0]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t* rc = r[c & 1];
+          tmem_wait_ld();
+          if (c + 1 < 4) tmem_ld32(tS + 32 * (c + 1), r[(c + 1) & 1]);
+          uint32_t pk[16];
+          if (chunk_kind[c] != 0) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float p0 = fast_exp2(fmaf(__uint_as_float(rc[e + 0]), sc, -msc));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(rc[e + 1]), sc, -msc));
+              pk[e >> 1] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) pk[e] = 0u;
+          }
+          tmem_st16(tS + 16 * c, pk);  // columns [16c, 16c+16): inside chunks already read
+        }
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(&sm.s_free[hh]);  // S_hh may be overwritten by the next key tile
-          mbar_arrive(&sm.p_full[hh]);
-        }
+        if (lane == 0) mbar_arrive(&sm.p_full[hh]);
         pr = pr_next;
         mk = mk_next;
       }
-      if (ok && (ok = mbar_wait(&sm.p_free[hh], (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status))) {
+      // the last PV product of this half (all earlier ones are complete by issue order)
+      if (ok && (ok = mbar_wait(&sm.o_full[hh], (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status))) {
         tc_fence_after();
-        const float inv = 1.f / row_sum;
         uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st;
         uint16_t* orow2 = orow + (int64_t)p.share_offset * p.o_sb;
+        uint32_t l16[16];
+        tmem_ld16(tO + kHeadDim, l16);  // row sum of the bf16 probabilities, from the ones block
+        tmem_wait_ld();
+        const float inv = 1.f / __uint_as_float(l16[0]);
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t r[32];
