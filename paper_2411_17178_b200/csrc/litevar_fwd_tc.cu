@@ -3,22 +3,25 @@
 //
 // One CTA handles two adjacent query tiles ("halves", 128 queries each) of one (head, batch row) and
 // walks the union of their live key-tile lists in plan order, so every K/V tile is staged once for
-// both halves.  384 threads in three warpgroups:
+// both halves.  640 threads:
 //   warp 0       TMA producer (one lane): Q of both halves, then K and V of every listed key tile into
 //                two rings of kStages tiles
 //   warp 1       TMEM allocation; one lane issues, per half h, O_h += P_h V (previous tile) and then
 //                S_h = Q_h K^T (next tile); the two halves alternate, so the tensor pipe works for one
 //                half while the other is in its softmax
-//   warps 4..7   softmax of half 0, warps 8..11 softmax of half 1: thread = query row (TMEM lane).
-//                Pass 1 over 32-key chunks: element mask (mixed chunks only, written back to TMEM) and
-//                the exact row max of the tile.  The row's reference max moves only when the tile
-//                exceeds it by more than 2^8; only then is the accumulator rescaled.  Pass 2:
-//                exponentials against the reference, P as packed bf16 written over the first half of
-//                S_h's own columns.  Chunks without a live key for the whole warp are skipped.
+//   warps 4..11  softmax of half 0, warps 12..19 softmax of half 1.  Two threads share a query row
+//                (TMEM lane): warps 4..7 / 12..15 take the first 64 keys of the tile, warps 8..11 /
+//                16..19 the last 64.  Pass 1 over 16-key chunks: element mask (mixed chunks only, written
+//                back to TMEM) and the row max of the thread's keys; the two partial maxima meet through
+//                shared memory and one mbarrier phase per tile.  The row's reference max moves only when
+//                the tile exceeds it by more than 2^8; only then is the accumulator rescaled.  Pass 2:
+//                exponentials against the reference, P as packed bf16 written over the first 32 of the
+//                thread's own 64 S columns.  Chunks without a live key for the whole warp are skipped.
 // Row sums come from the tensor pipe: the B operand of the PV product is V (64 columns) followed by a
 // block of ones (16 columns), so accumulator column 64 holds sum_t P[q,t] of the very bf16 weights the
 // output uses; no per-element add is issued.
-// TMEM columns: S_0/P_0 [0,128)  S_1/P_1 [128,256)  O_0 [256,336)  O_1 [336,416).
+// TMEM columns: S_0 [0,128)  S_1 [128,256)  O_0 [256,336)  O_1 [336,416); P_h for keys [0,64) lies in
+// S_h columns [0,32), for keys [64,128) in S_h columns [64,96).
 //
 // Every wait is bounded: when a wait runs out the CTA raises the plan's status word, drains its
 // outstanding copies, frees its TMEM and returns.
@@ -35,7 +38,7 @@ namespace litevar {
 namespace {
 
 constexpr int kStages = 4;
-constexpr int kThreads = 384;
+constexpr int kThreads = 640;
 constexpr uint32_t kTileBytes = kBlockN * kHeadDim * 2;  // 16 KB: 128 rows of 128 B
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;  // + 128 / kOutCols per half; P_h overlays S_h
@@ -51,7 +54,8 @@ struct SharedStorage {
   alignas(1024) uint8_t ones[kTileBytes];  // bf16 1.0 everywhere: second N block of the PV product's B operand
   alignas(8) uint64_t q_full;
   uint64_t k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
-  uint64_t s_full[2], p_full[2], o_full[2];
+  uint64_t s_full[2], p_full[2], o_full[2], x_full[2];
+  float xmax[2][2][2][kBlockM];  // [tile parity][half][key half][row]: partial row maxima of a tile
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -204,6 +208,11 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -269,8 +278,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.p_full[i], 4);
+      mbar_init(&sm.p_full[i], 8);
       mbar_init(&sm.o_full[i], 1);
+      mbar_init(&sm.x_full[i], 8);
     }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -371,8 +381,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
             tc_fence_after();
 #pragma unroll
-            for (int kk = 0; kk < kBlockN / 16; ++kk)  // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns
-              mma_ts(tmem + kColO + kOutCols * hh, tmem + kColS + 128 * hh + 8 * kk,
+            for (int kk = 0; kk < kBlockN / 16; ++kk)  // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns per step, key half 1 starts at S column 64
+              mma_ts(tmem + kColO + kOutCols * hh, tmem + kColS + 128 * hh + 8 * kk + (kk >= 4 ? 32 : 0),
                      v_desc + (uint64_t)(2048 >> 4) * kk, kIdescPV, (n_pv[hh] > 0 || kk > 0) ? 1u : 0u);
             mma_commit(&sm.o_full[hh]);
             ++n_pv[hh];
@@ -396,7 +406,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue of one half
-    const int hh = (warp - 4) >> 2;
+    const int hh = (warp - 4) >> 3;        // query half
+    const int sub = ((warp - 4) >> 2) & 1;  // key half of every tile this thread works on
     const int qt = hh ? qt1 : qt0;
     const int pbeg = hh ? beg1 : beg0;
     const int n_tiles = (hh ? end1 : end0) - pbeg;
@@ -405,24 +416,27 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       const int m = lane_group * 32 + lane;
       const int q = qt * kBlockM + m;
       const uint32_t tlane = tmem + ((uint32_t)(lane_group * 32) << 16);
-      const uint32_t tS = tlane + kColS + 128 * hh, tO = tlane + kColO + kOutCols * hh;
+      const uint32_t tS = tlane + kColS + 128 * hh + 64 * sub;  // this thread's 64 score columns
+      const uint32_t tO = tlane + kColO + kOutCols * hh;
       const float sc = p.sm_scale * 1.4426950408889634f;
       float row_max = -INFINITY;  // the score the stored probabilities refer to
       bool ok = true;
       Pair pr = sd.pairs[pbeg];
-      uint4 mk = make_uint4(~0u, ~0u, ~0u, ~0u);
-      if (pr.mask_block >= 0) mk = __ldg(&sd.mask[(size_t)pr.mask_block * kBlockM + m]);
+      uint2 mk = make_uint2(~0u, ~0u);
+      if (pr.mask_block >= 0)
+        mk = __ldg(reinterpret_cast<const uint2*>(&sd.mask[(size_t)pr.mask_block * kBlockM + m]) + sub);
       for (int j = 0; j < n_tiles; ++j) {
         // next pair's mask words travel while this tile is processed
         Pair pr_next = pr;
-        uint4 mk_next = make_uint4(~0u, ~0u, ~0u, ~0u);
+        uint2 mk_next = make_uint2(~0u, ~0u);
         if (j + 1 < n_tiles) {
           pr_next = sd.pairs[pbeg + j + 1];
-          if (pr_next.mask_block >= 0) mk_next = __ldg(&sd.mask[(size_t)pr_next.mask_block * kBlockM + m]);
+          if (pr_next.mask_block >= 0)
+            mk_next = __ldg(reinterpret_cast<const uint2*>(&sd.mask[(size_t)pr_next.mask_block * kBlockM + m]) + sub);
         }
         const bool partial = pr.mask_block >= 0;
-        const uint32_t wbits[4] = {mk.x, mk.y, mk.z, mk.w};
-        // per 32-key chunk, uniform over the warp: 0 = no live key (skipped), 1 = mixed, 2 = all live
+        // per 16-key chunk, uniform over the warp: 0 = no live key (skipped), 1 = mixed, 2 = all live
+        uint32_t wbits[4] = {mk.x & 0xffffu, mk.x >> 16, mk.y & 0xffffu, mk.y >> 16};
         int chunk_kind[4];
         bool any_mixed = false;
 #pragma unroll
@@ -430,74 +444,82 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
           chunk_kind[c] = 2;
           if (partial)
             chunk_kind[c] = !__any_sync(0xffffffffu, wbits[c] != 0u) ? 0
-                            : (__all_sync(0xffffffffu, wbits[c] == 0xffffffffu) ? 2 : 1);
+                            : (__all_sync(0xffffffffu, wbits[c] == 0xffffu) ? 2 : 1);
           any_mixed |= chunk_kind[c] == 1;
         }
         // S_hh(j) complete; in issue order this also means the PV product of tile j-1 is complete
         if (!(ok = mbar_wait(&sm.s_full[hh], (uint32_t)(j & 1), abort_flag, p.status))) break;
         tc_fence_after();
-        uint32_t r[2][32];
-        // ---- pass 1: mask the mixed chunks (written back) and take the row max of the tile
+        uint32_t r[2][16];
+        // ---- pass 1: mask the mixed chunks (written back) and take the max of this thread's 64 keys
         float mx0 = -INFINITY, mx1 = -INFINITY;
-        tmem_ld32(tS, r[0]);
+        tmem_ld16(tS, r[0]);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t* rc = r[c & 1];
           tmem_wait_ld();
-          if (c + 1 < 4) tmem_ld32(tS + 32 * (c + 1), r[(c + 1) & 1]);
+          if (c + 1 < 4) tmem_ld16(tS + 16 * (c + 1), r[(c + 1) & 1]);
           if (chunk_kind[c] == 0) continue;
           if (chunk_kind[c] == 1) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
+            for (int e = 0; e < 16; ++e)
               if (!((wbits[c] >> e) & 1u)) rc[e] = 0xff800000u;  // -inf
-            tmem_st32(tS + 32 * c, rc);
+            tmem_st16(tS + 16 * c, rc);
           }
 #pragma unroll
-          for (int e = 0; e < 32; e += 4) {
+          for (int e = 0; e < 16; e += 4) {
             mx0 = max3(mx0, __uint_as_float(rc[e + 0]), __uint_as_float(rc[e + 1]));
             mx1 = max3(mx1, __uint_as_float(rc[e + 2]), __uint_as_float(rc[e + 3]));
           }
         }
-        const float tile_max = fmaxf(mx0, mx1);
+        // the two threads of a row exchange their maxima
+        float tile_max = fmaxf(mx0, mx1);
+        sm.xmax[j & 1][hh][sub][m] = tile_max;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.x_full[hh]);
+        if (!(ok = mbar_wait(&sm.x_full[hh], (uint32_t)(j & 1), abort_flag, p.status))) break;
+        tile_max = fmaxf(tile_max, sm.xmax[j & 1][hh][sub ^ 1][m]);
         // the reference max moves only when the tile exceeds it by more than the threshold
         float alpha = 1.f;
         if ((tile_max - row_max) * sc > kRescaleThreshold) {  // false for tile_max = -inf, true for row_max = -inf
           if (row_max != -INFINITY) alpha = fast_exp2((row_max - tile_max) * sc);
           row_max = tile_max;
         }
-        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // accumulator and row sum follow the reference
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+          // accumulator and row sum follow the reference: columns [0,48) here, [48,80) in the partner thread
           uint32_t o[16];
 #pragma unroll
-          for (int c = 0; c < kOutCols / 16; ++c) {
-            tmem_ld16(tO + 16 * c, o);
+          for (int c = 0; c < 3 - sub; ++c) {
+            const uint32_t col = 48 * sub + 16 * c;
+            tmem_ld16(tO + col, o);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st16(tO + 16 * c, o);
+            tmem_st16(tO + col, o);
           }
         }
         if (any_mixed) tmem_wait_st();  // the masked scores are read back below
-        // ---- pass 2: probabilities against the reference; P (packed bf16) over S_hh's first 64 columns
+        // ---- pass 2: probabilities against the reference; P (packed bf16) over this thread's first 32 columns
         const float msc = row_max == -INFINITY ? 0.f : row_max * sc;
-        tmem_ld32(tS, r[0]);
+        tmem_ld16(tS, r[0]);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t* rc = r[c & 1];
           tmem_wait_ld();
-          if (c + 1 < 4) tmem_ld32(tS + 32 * (c + 1), r[(c + 1) & 1]);
-          uint32_t pk[16];
+          if (c + 1 < 4) tmem_ld16(tS + 16 * (c + 1), r[(c + 1) & 1]);
+          uint32_t pk[8];
           if (chunk_kind[c] != 0) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
+            for (int e = 0; e < 16; e += 2) {
               const float p0 = fast_exp2(fmaf(__uint_as_float(rc[e + 0]), sc, -msc));
               const float p1 = fast_exp2(fmaf(__uint_as_float(rc[e + 1]), sc, -msc));
               pk[e >> 1] = pack_bf16(p0, p1);
             }
           } else {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) pk[e] = 0u;
+            for (int e = 0; e < 8; ++e) pk[e] = 0u;
           }
-          tmem_st16(tS + 16 * c, pk);  // columns [16c, 16c+16): inside chunks already read
+          tmem_st8(tS + 8 * c, pk);  // columns [8c, 8c+8) of this thread's 64: inside chunks already read
         }
         tmem_wait_st();
         tc_fence_before();
@@ -509,28 +531,25 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       // the last PV product of this half (all earlier ones are complete by issue order)
       if (ok && (ok = mbar_wait(&sm.o_full[hh], (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status))) {
         tc_fence_after();
-        uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st;
+        // this thread stores output columns [32 sub, 32 sub + 32) of its row
+        uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st + 32 * sub;
         uint16_t* orow2 = orow + (int64_t)p.share_offset * p.o_sb;
         uint32_t l16[16];
         tmem_ld16(tO + kHeadDim, l16);  // row sum of the bf16 probabilities, from the ones block
+        uint32_t r[32];
+        tmem_ld32(tO + 32 * sub, r);
         tmem_wait_ld();
         const float inv = 1.f / __uint_as_float(l16[0]);
+        if (q < p.n_k) {
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tO + 32 * c, r);
-          tmem_wait_ld();
-          if (q < p.n_k) {
-#pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              uint4 o4;
-              o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
-              o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-              o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-              o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-              *reinterpret_cast<uint4*>(orow + 32 * c + e) = o4;
-              if (p.share_offset > 0) *reinterpret_cast<uint4*>(orow2 + 32 * c + e) = o4;
-            }
+          for (int e = 0; e < 32; e += 8) {
+            uint4 o4;
+            o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
+            o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+            o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+            o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + e) = o4;
+            if (p.share_offset > 0) *reinterpret_cast<uint4*>(orow2 + e) = o4;
           }
         }
       }
