@@ -46,6 +46,13 @@ typedef enum {
  * the flattened attention map. */
 enum { LITEVAR_WINDOW_SQUARE = 0, LITEVAR_WINDOW_BAND = 1 };
 
+/* Tile geometry of the plan.  RASTER: every query and key tile is 128 consecutive tokens.  PATCH:
+ * a query tile is an 8 x 16 patch of the current scale's grid and the keys of the larger scales
+ * are tiled in 8 x 16 patches of their own grids (grid-aligned), so that a 2-D window leaves whole
+ * tiles dead; the coarse scales in front stay raster.  AUTO picks PATCH for steps whose grid side is
+ * at least 48 (key scales of side >= 32 in patches, at most 8 of them) and RASTER otherwise. */
+enum { LITEVAR_TILING_AUTO = 0, LITEVAR_TILING_RASTER = 1, LITEVAR_TILING_PATCH = 2 };
+
 /* Window specification (paper Section 2: one window width per part of the step-k map; the
  * first parts stay global, "MDWA implementation details"). */
 typedef struct {
@@ -57,6 +64,7 @@ typedef struct {
                                -1 = whole part live; copied at plan time; entries with j > k ignored */
   int32_t n_sets;           /* number of window tables (paper: widths are chosen per head); >= 1 */
   const int32_t* head_to_set; /* host [n_heads], values in [0, n_sets); NULL = all heads use set 0 */
+  int32_t tiling;           /* LITEVAR_TILING_*; changes the tile lists and the speed, never the result */
 } litevar_window_t;
 
 /* CFG sharing (paper Section 3): at a shared step the unconditional half of the batch
@@ -175,9 +183,12 @@ litevar_status_t litevar_plan_tile_counts(const litevar_plan_t* plan, int32_t st
 
 /*
  * Copy the step-k tile plan to host arrays sized from litevar_plan_tile_counts (any may be NULL):
- *   q_tile_geom   [n_q_tiles][4]   {first token, slots, row stride, columns}: slot m is token
- *                                  first + (m / columns) * row_stride + (m % columns)
- *   key_tile_geom [n_key_tiles][4] same, tokens index the K/V cache
+ *   q_tile_geom   [n_q_tiles][5]   {first token, columns, row stride, valid rows, valid columns}: slot m
+ *                                  (0 <= m < 128) sits at row m / columns, column m % columns of the tile; it
+ *                                  holds token first + row * row_stride + column when row < valid rows and
+ *                                  column < valid columns, and is padding otherwise (raster tiles: one row of
+ *                                  128 columns; patch tiles: 8 rows of 16 columns, row stride = grid side)
+ *   key_tile_geom [n_key_tiles][5] same, tokens index the K/V cache
  *   row_ptr       [n_q_tiles + 1]  CSR offsets into the pair arrays
  *   pair_key_tile [n_pairs]        key tile of each live pair, ascending inside a query tile
  *   pair_is_full  [n_pairs]        1 = every slot pair live (no element mask), 0 = partial

@@ -21,6 +21,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "EMPTY_ROW", 4: 
                 7: "DEVICE_TIMEOUT"}
 WINDOW_SQUARE, WINDOW_BAND = 0, 1
 KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
+TILING_AUTO, TILING_RASTER, TILING_PATCH = 0, 1, 2
 
 EXPORTS = (
     "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_static", "litevar_plan_stats", "litevar_plan_tile_counts",
@@ -40,7 +41,7 @@ class _Window(ctypes.Structure):
     _fields_ = [("shape", ctypes.c_int32), ("n_global_scales", ctypes.c_int32),
                 ("rho_num", ctypes.c_int32), ("rho_den", ctypes.c_int32),
                 ("radius", ctypes.POINTER(ctypes.c_int32)), ("n_sets", ctypes.c_int32),
-                ("head_to_set", ctypes.POINTER(ctypes.c_int32))]
+                ("head_to_set", ctypes.POINTER(ctypes.c_int32)), ("tiling", ctypes.c_int32)]
 
 
 class _Share(ctypes.Structure):
@@ -125,7 +126,7 @@ class Plan:
 
     def __init__(self, scales: Sequence[int], n_heads: int, head_dim: int = 64, sm_scale: float = 0.0,
                  shape: int = WINDOW_SQUARE, n_global_scales: int = 3, rho=(1, 4), radius=None,
-                 n_sets: int = 1, head_to_set=None, share_steps=None, stream=None):
+                 n_sets: int = 1, head_to_set=None, share_steps=None, stream=None, tiling: int = TILING_AUTO):
         lib = load()
         self._lib = lib
         self.scales = tuple(int(s) for s in scales)
@@ -136,6 +137,7 @@ class Plan:
         win.shape, win.n_global_scales = int(shape), int(n_global_scales)
         win.rho_num, win.rho_den = int(rho[0]), int(rho[1])
         win.n_sets = self.n_sets
+        win.tiling = int(tiling)
         keep = []
         if radius is not None:
             arr = np.ascontiguousarray(np.asarray(radius, dtype=np.int32).reshape(self.n_sets, K, K))
@@ -201,8 +203,8 @@ class Plan:
 
     def export_tiles(self, step_k: int, set_index: int = 0) -> dict:
         nq, nk, npairs = self.tile_counts(step_k, set_index)
-        qg = np.zeros((nq, 4), np.int32)
-        kg = np.zeros((nk, 4), np.int32)
+        qg = np.zeros((nq, 5), np.int32)
+        kg = np.zeros((nk, 5), np.int32)
         rp = np.zeros(nq + 1, np.int32)
         pk = np.zeros(max(npairs, 1), np.int32)
         pf = np.zeros(max(npairs, 1), np.uint8)

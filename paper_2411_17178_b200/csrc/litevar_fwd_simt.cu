@@ -17,15 +17,34 @@ constexpr int kWarpsPerBlock = 4;
 
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
 
+// Cache row of slot n of key tile `kt` (any row for a padding slot: its mask bit is never set).
+__device__ __forceinline__ int key_slot_row(const FwdParams& p, int kt, int n) {
+  if (p.key_geom == nullptr) return kt * kBlockN + n;
+  const TileGeom g = p.key_geom[kt];
+  if (g.scale < 0) return g.a + n;
+  const int s_j = p.patch_scale[g.map_slot];
+  return p.patch_off[g.map_slot] + (g.a + n / kPatchCols) * s_j + g.b + n % kPatchCols;
+}
+
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) fwd_simt_kernel(FwdParams p) {
   __shared__ float q_sh[kWarpsPerBlock][kHeadDim];
   __shared__ float p_sh[kWarpsPerBlock][kBlockN];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q = blockIdx.x * kWarpsPerBlock + warp;
+  const int slot = blockIdx.x * kWarpsPerBlock + warp;  // one warp per query slot of the tile plan
   const int h = blockIdx.y, b = blockIdx.z;
-  if (q >= p.n_k) return;  // whole warp
+  const int qt = slot / kBlockM, m = slot % kBlockM;
+  int q = slot;
+  if (p.q_geom != nullptr) {
+    const TileGeom g = p.q_geom[qt];
+    if (g.scale < 0) {
+      q = g.a + m;
+    } else {
+      const int r = g.a + m / kPatchCols, c = g.b + m % kPatchCols;
+      q = (r < p.s_k && c < p.s_k) ? r * p.s_k + c : p.n_k;
+    }
+  }
+  if (q >= p.n_k) return;  // padding slot (whole warp)
   const SetDesc sd = p.sets[p.head_to_set ? p.head_to_set[h] : 0];
-  const int qt = q / kBlockM, m = q % kBlockM;
 
   const uint16_t* qrow = p.q + b * p.q_sb + h * p.q_sh + (int64_t)q * p.q_st;
   q_sh[warp][lane] = bf16_bits_to_float(qrow[lane]);
@@ -42,14 +61,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fwd_simt_kernel(FwdParams
                                     : sd.mask[(size_t)pr.mask_block * kBlockM + m];
     const uint32_t bits[4] = {bits4.x, bits4.y, bits4.z, bits4.w};
     if ((bits[0] | bits[1] | bits[2] | bits[3]) == 0u) continue;
-    const int t0 = pr.key_tile * kBlockN;
     float s[4];
     float tile_max = -INFINITY;
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
       s[w] = -INFINITY;
       if ((bits[w] >> lane) & 1u) {
-        const uint4* krow = reinterpret_cast<const uint4*>(kbase + (int64_t)(t0 + w * 32 + lane) * p.k_st);
+        const uint4* krow =
+            reinterpret_cast<const uint4*>(kbase + (int64_t)key_slot_row(p, pr.key_tile, w * 32 + lane) * p.k_st);
         float dot = 0.f;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -89,7 +108,8 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fwd_simt_kernel(FwdParams
         int n = __ffs(bw) - 1;
         bw &= bw - 1;
         float pv = p_sh[warp][w * 32 + n];
-        uint32_t vv = *reinterpret_cast<const uint32_t*>(vbase + (int64_t)(t0 + w * 32 + n) * p.v_st + 2 * lane);
+        uint32_t vv = *reinterpret_cast<const uint32_t*>(
+            vbase + (int64_t)key_slot_row(p, pr.key_tile, w * 32 + n) * p.v_st + 2 * lane);
         acc0 = fmaf(pv, __uint_as_float(vv << 16), acc0);
         acc1 = fmaf(pv, __uint_as_float(vv & 0xffff0000u), acc1);
       }
@@ -109,8 +129,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fwd_simt_kernel(FwdParams
 }  // namespace
 
 cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
-  (void)n_q_tiles;
-  dim3 grid((unsigned)((p.n_k + kWarpsPerBlock - 1) / kWarpsPerBlock), (unsigned)p.n_heads,
+  dim3 grid((unsigned)(n_q_tiles * (kBlockM / kWarpsPerBlock)), (unsigned)p.n_heads,
             (unsigned)p.batch_computed);
   fwd_simt_kernel<<<grid, kWarpsPerBlock * 32, 0, stream>>>(p);
   return cudaGetLastError();

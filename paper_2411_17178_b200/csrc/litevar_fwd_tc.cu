@@ -29,6 +29,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cstring>
 #include <mutex>
 
 #include "litevar_internal.h"
@@ -144,6 +145,58 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, i
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, const void* src, int c0, int c1, int c2, int c3,
+                                             int c4) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+               : "memory");
+}
+
+// Tensor maps of one launch.  q and o are rank 4 (raster query tiles) or rank 5 (patch query tiles); kr/vr
+// cover the raster prefix of the cache; k2/v2[i] cover the grid of the i-th key scale tiled in patches.
+struct TensorMaps {
+  CUtensorMap q, o, kr, vr;
+  CUtensorMap k2[kMaxPatchScales], v2[kMaxPatchScales];
+};
+
+// Loads of one query / key tile according to its geometry.
+__device__ __forceinline__ void load_q_tile(void* dst, const TensorMaps& tm, const FwdParams& p, int qt, int h, int b,
+                                            uint64_t* bar) {
+  if (p.q_geom == nullptr) {
+    tma_load_4d(dst, &tm.q, 0, qt * kBlockM, h, b, bar);
+    return;
+  }
+  const TileGeom g = p.q_geom[qt];
+  if (g.scale < 0)
+    tma_load_4d(dst, &tm.q, 0, g.a, h, b, bar);
+  else
+    tma_load_5d(dst, &tm.q, 0, g.b, g.a, h, b, bar);
+}
+__device__ __forceinline__ void load_kv_tile(void* dst, const CUtensorMap* raster, const CUtensorMap* patch,
+                                             const FwdParams& p, int kt, int h, int b, uint64_t* bar) {
+  if (p.key_geom == nullptr) {
+    tma_load_4d(dst, raster, 0, kt * kBlockN, h, b, bar);
+    return;
+  }
+  const TileGeom g = p.key_geom[kt];
+  if (g.scale < 0)
+    tma_load_4d(dst, raster, 0, g.a, h, b, bar);
+  else
+    tma_load_5d(dst, patch + g.map_slot, 0, g.b, g.a, h, b, bar);
+}
+
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {
   asm volatile(
@@ -257,8 +310,7 @@ struct UnionWalk {
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-              const __grid_constant__ CUtensorMap tm_v, FwdParams p, int n_q_tiles) {
+fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ FwdParams p, int n_q_tiles) {
   extern __shared__ uint8_t smem_raw[];
   SharedStorage& sm = *reinterpret_cast<SharedStorage*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -302,6 +354,24 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   const SetDesc sd = p.sets[p.head_to_set ? p.head_to_set[h] : 0];
   const int beg0 = __ldg(&sd.row_ptr[qt0]), end0 = __ldg(&sd.row_ptr[qt0 + 1]);
   const int beg1 = end0, end1 = has1 ? __ldg(&sd.row_ptr[qt1 + 1]) : end0;
+  // The producer lane (it initialised the barriers itself) starts the first copies before the set-up
+  // barrier: Q of both halves, K and V of the first listed key tile.
+  UnionWalk pw;
+  int p_issued = 0;
+  if (threadIdx.x == 0 && end1 > beg0) {
+    const bool ld0 = end0 > beg0, ld1 = end1 > beg1;
+    mbar_expect_tx(&sm.q_full, (ld0 ? kTileBytes : 0u) + (ld1 ? kTileBytes : 0u));
+    if (ld0) load_q_tile(sm.q[0], tm, p, qt0, h, b, &sm.q_full);
+    if (ld1) load_q_tile(sm.q[1], tm, p, qt1, h, b, &sm.q_full);
+    pw.init(sd.pairs, beg0, end0, beg1, end1);
+    bool l0, l1;
+    const int kt = pw.next(l0, l1);
+    mbar_expect_tx(&sm.k_full[0], kTileBytes);
+    load_kv_tile(sm.k[0], &tm.kr, tm.k2, p, kt, h, b, &sm.k_full[0]);
+    mbar_expect_tx(&sm.v_full[0], kTileBytes);
+    load_kv_tile(sm.v[0], &tm.vr, tm.v2, p, kt, h, b, &sm.v_full[0]);
+    p_issued = 1;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -310,20 +380,14 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   if (warp < 4) {
     if (warp == 0 && lane == 0 && end1 > beg0) {
       // ---------------------------------------------------------------- TMA producer
-      const bool ld0 = end0 > beg0, ld1 = end1 > beg1;
-      mbar_expect_tx(&sm.q_full, (ld0 ? kTileBytes : 0u) + (ld1 ? kTileBytes : 0u));
-      if (ld0) tma_load_4d(sm.q[0], &tm_q, 0, qt0 * kBlockM, h, b, &sm.q_full);
-      if (ld1) tma_load_4d(sm.q[1], &tm_q, 0, qt1 * kBlockM, h, b, &sm.q_full);
-      UnionWalk w;
-      w.init(sd.pairs, beg0, end0, beg1, end1);
-      int issued = 0;
-      for (int i = 0; w.has(); ++i) {
+      int issued = p_issued;
+      for (int i = p_issued; pw.has(); ++i) {
         bool l0, l1;
-        const int t0 = w.next(l0, l1) * kBlockN;
+        const int kt = pw.next(l0, l1);
         const int s = i % kStages, n = i / kStages;
         if (n > 0 && !mbar_wait(&sm.k_free[s], (uint32_t)((n - 1) & 1), abort_flag, p.status)) break;
         mbar_expect_tx(&sm.k_full[s], kTileBytes);
-        tma_load_4d(sm.k[s], &tm_k, 0, t0, h, b, &sm.k_full[s]);
+        load_kv_tile(sm.k[s], &tm.kr, tm.k2, p, kt, h, b, &sm.k_full[s]);
         if (n > 0 && !mbar_wait(&sm.v_free[s], (uint32_t)((n - 1) & 1), abort_flag, p.status)) {
           // the K copy just issued is still in flight
           const unsigned long long ts = global_ns();
@@ -332,7 +396,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
           break;
         }
         mbar_expect_tx(&sm.v_full[s], kTileBytes);
-        tma_load_4d(sm.v[s], &tm_v, 0, t0, h, b, &sm.v_full[s]);
+        load_kv_tile(sm.v[s], &tm.vr, tm.v2, p, kt, h, b, &sm.v_full[s]);
         issued = i + 1;
       }
       if (*abort_flag) {
@@ -414,7 +478,6 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     if (n_tiles > 0) {
       const int lane_group = warp & 3;  // TMEM lanes this warp may touch: 32*lane_group .. +31
       const int m = lane_group * 32 + lane;
-      const int q = qt * kBlockM + m;
       const uint32_t tlane = tmem + ((uint32_t)(lane_group * 32) << 16);
       const uint32_t tS = tlane + kColS + 128 * hh + 64 * sub;  // this thread's 64 score columns
       const uint32_t tO = tlane + kColO + kOutCols * hh;
@@ -531,26 +594,45 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       // the last PV product of this half (all earlier ones are complete by issue order)
       if (ok && (ok = mbar_wait(&sm.o_full[hh], (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status))) {
         tc_fence_after();
-        // this thread stores output columns [32 sub, 32 sub + 32) of its row
-        uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st + 32 * sub;
-        uint16_t* orow2 = orow + (int64_t)p.share_offset * p.o_sb;
+        // normalised bf16 row into the half's Q buffer (its last reader, S_hh of the last tile, is done),
+        // in the 128-byte swizzle the output tensor map expects; one lane then stores the whole tile
         uint32_t l16[16];
         tmem_ld16(tO + kHeadDim, l16);  // row sum of the bf16 probabilities, from the ones block
         uint32_t r[32];
         tmem_ld32(tO + 32 * sub, r);
         tmem_wait_ld();
         const float inv = 1.f / __uint_as_float(l16[0]);
-        if (q < p.n_k) {
+        uint8_t* srow = sm.q[hh] + m * 128;
 #pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 o4;
-            o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
-            o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-            o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-            o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + e) = o4;
-            if (p.share_offset > 0) *reinterpret_cast<uint4*>(orow2 + e) = o4;
+        for (int e = 0; e < 32; e += 8) {
+          uint4 o4;
+          o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
+          o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+          o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+          o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+          const int chunk = 4 * sub + (e >> 3);
+          *reinterpret_cast<uint4*>(srow + ((chunk ^ (m & 7)) << 4)) = o4;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.x_full[hh]);
+        if (warp == 4 + 8 * hh && lane == 0 &&
+            mbar_wait(&sm.x_full[hh], (uint32_t)(n_tiles & 1), abort_flag, p.status)) {
+          const int nb = p.share_offset > 0 ? 2 : 1;  // under CFG sharing the tile also goes to row b + B
+          for (int i = 0; i < nb; ++i) {
+            const int bo = b + i * p.share_offset;
+            if (p.q_geom == nullptr) {
+              tma_store_4d(&tm.o, sm.q[hh], 0, qt * kBlockM, h, bo);
+            } else {
+              const TileGeom g = p.q_geom[qt];
+              if (g.scale < 0)
+                tma_store_4d(&tm.o, sm.q[hh], 0, g.a, h, bo);
+              else
+                tma_store_5d(&tm.o, sm.q[hh], 0, g.b, g.a, h, bo);
+            }
           }
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         }
       }
     }
@@ -587,10 +669,11 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // Rank-4 map over a [batch, head, token, 64] bf16 tensor with element strides; box = 128 tokens x 64.
-bool encode_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t heads, int64_t batch, int64_t st,
-                int64_t sh, int64_t sb) {
+bool encode_raster(CUtensorMap* tm, const void* base, int64_t rows, int64_t heads, int64_t batch, int64_t st,
+                   int64_t sh, int64_t sb) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
+  if (rows < 1) rows = 1;  // no raster tile will use this map
   // a dimension of extent 1 may come with any stride; give it a valid one
   if (heads == 1 && sh < kHeadDim) sh = st * rows;
   if (batch == 1 && sb < kHeadDim) sb = sh * heads;
@@ -599,6 +682,26 @@ bool encode_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t heads, 
   cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)kBlockN, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Rank-5 map over the side x side grid of one scale inside a [batch, head, token, 64] tensor: dimensions
+// (64, column, row, head, batch); box = 8 rows x 16 columns x 64, i.e. 128 rows of 128 B in shared memory in
+// row-major patch order.  Cells outside the grid read as zero and are not written.
+bool encode_patch(CUtensorMap* tm, const void* base, int64_t first_token, int64_t side, int64_t heads,
+                  int64_t batch, int64_t st, int64_t sh, int64_t sb) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  if (heads == 1 && sh < kHeadDim) sh = st * side * side;
+  if (batch == 1 && sb < kHeadDim) sb = sh * heads;
+  const uint16_t* origin = static_cast<const uint16_t*>(base) + first_token * st;
+  cuuint64_t gdim[5] = {(cuuint64_t)kHeadDim, (cuuint64_t)side, (cuuint64_t)side, (cuuint64_t)heads, (cuuint64_t)batch};
+  cuuint64_t gstr[4] = {(cuuint64_t)st * 2, (cuuint64_t)(st * side) * 2, (cuuint64_t)sh * 2, (cuuint64_t)sb * 2};
+  cuuint32_t box[5] = {(cuuint32_t)kHeadDim, (cuuint32_t)kPatchCols, (cuuint32_t)kPatchRows, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<uint16_t*>(origin), gdim, gstr, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -614,13 +717,26 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
     attr_err = cudaFuncSetAttribute(fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   });
   if (attr_err != cudaSuccess) return LITEVAR_ERR_CUDA;
-  CUtensorMap tm_q, tm_k, tm_v;
-  if (!encode_map(&tm_q, p.q, p.n_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb) ||
-      !encode_map(&tm_k, p.k, p.L_k, p.n_heads, p.batch_computed, p.k_st, p.k_sh, p.k_sb) ||
-      !encode_map(&tm_v, p.v, p.L_k, p.n_heads, p.batch_computed, p.v_st, p.v_sh, p.v_sb))
-    return LITEVAR_ERR_INVALID_ARG;
+  TensorMaps tm;
+  memset(&tm, 0, sizeof(tm));
+  const int64_t out_rows = p.batch_computed + p.share_offset;
+  bool ok;
+  if (p.q_patch)
+    ok = encode_patch(&tm.q, p.q, 0, p.s_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb) &&
+         encode_patch(&tm.o, p.out, 0, p.s_k, p.n_heads, out_rows, p.o_st, p.o_sh, p.o_sb);
+  else
+    ok = encode_raster(&tm.q, p.q, p.n_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb) &&
+         encode_raster(&tm.o, p.out, p.n_k, p.n_heads, out_rows, p.o_st, p.o_sh, p.o_sb);
+  ok = ok && encode_raster(&tm.kr, p.k, p.raster_len, p.n_heads, p.batch_computed, p.k_st, p.k_sh, p.k_sb) &&
+       encode_raster(&tm.vr, p.v, p.raster_len, p.n_heads, p.batch_computed, p.v_st, p.v_sh, p.v_sb);
+  for (int i = 0; ok && i < p.n_patch_scales; ++i)
+    ok = encode_patch(&tm.k2[i], p.k, p.patch_off[i], p.patch_scale[i], p.n_heads, p.batch_computed, p.k_st, p.k_sh,
+                      p.k_sb) &&
+         encode_patch(&tm.v2[i], p.v, p.patch_off[i], p.patch_scale[i], p.n_heads, p.batch_computed, p.v_st, p.v_sh,
+                      p.v_sb);
+  if (!ok) return LITEVAR_ERR_INVALID_ARG;
   dim3 grid((unsigned)((n_q_tiles + 1) / 2), (unsigned)p.n_heads, (unsigned)p.batch_computed);
-  fwd_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p, n_q_tiles);
+  fwd_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tm, p, n_q_tiles);
   if (cudaGetLastError() != cudaSuccess) return LITEVAR_ERR_CUDA;
   return LITEVAR_OK;
 }

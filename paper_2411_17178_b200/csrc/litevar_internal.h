@@ -31,6 +31,15 @@ struct Pair {
   int32_t mask_block;
 };
 
+// Geometry of one query or key tile (128 slots).  Raster: scale < 0, slot m is token a + m (query tiles:
+// token of the current scale; key tiles: cache row, valid below the end of the raster prefix).  Patch:
+// scale = 0-based scale index, slot m is grid cell (a + m / kPatchCols, b + m % kPatchCols) of that scale.
+struct TileGeom {
+  int32_t scale, a, b, map_slot;  // map_slot: index of the scale's tensor maps in the forward kernel (patch tiles)
+};
+constexpr int kPatchRows = 8, kPatchCols = 16;  // kPatchRows * kPatchCols == 128
+constexpr int kMaxPatchScales = 8;              // key scales that can be tiled in 2-D patches
+
 // Device-visible tile plan of one (step, window set).
 struct SetDesc {
   const int32_t* row_ptr;  // [n_q_tiles + 1]
@@ -50,6 +59,13 @@ struct StepSet {
 struct Step {
   int32_t s_k = 0, n_k = 0, L_k = 0, n_q_tiles = 0, n_key_tiles = 0;
   bool share = false;
+  bool q_patch = false;       // query tiles are 2-D patches of the current scale's grid
+  int32_t first_patch = 0;    // key scales with 0-based index >= first_patch are tiled in patches (== step count: none)
+  int32_t raster_len = 0;     // cache rows [0, raster_len) are covered by raster key tiles
+  int32_t n_raster_tiles = 0;
+  litevar::TileGeom* d_q_geom = nullptr;    // [n_q_tiles]
+  litevar::TileGeom* d_key_geom = nullptr;  // [n_key_tiles]
+  std::vector<litevar::TileGeom> q_geom, key_geom;  // host copies
   std::vector<StepSet> sets;
   SetDesc* d_sets = nullptr;  // [n_sets]
 };
@@ -67,6 +83,16 @@ struct FwdParams {
   int64_t v_sb, v_sh, v_st;
   int64_t o_sb, o_sh, o_st;
   int32_t n_k, L_k, n_heads;
+  // tile geometry; q_geom == nullptr: raster tiles everywhere (tile i = tokens [128 i, 128 i + 128))
+  const TileGeom* q_geom;
+  const TileGeom* key_geom;
+  int32_t s_k;              // side of the current scale's grid
+  int32_t q_patch;          // query tiles are patches (host: rank of the Q and output tensor maps)
+  int32_t raster_len;       // cache rows covered by raster key tiles (L_k when there are no patch tiles)
+  int32_t first_patch;      // first key scale (0-based) tiled in patches
+  int32_t n_patch_scales;   // number of such scales (<= kMaxPatchScales)
+  int32_t patch_scale[kMaxPatchScales];  // their grid sides
+  int32_t patch_off[kMaxPatchScales];    // their first cache rows
   int32_t batch_computed;       // rows the grid covers (B when shared, else 2B)
   int32_t share_offset;         // B when the step is shared (second store at row b + B), else 0
   float sm_scale;
@@ -82,7 +108,7 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
 
 struct litevar_plan {
   litevar::Schedule sched;
-  int32_t n_heads = 0, n_sets = 1, shape = 0, n_global = 0, rho_num = 1, rho_den = 4;
+  int32_t n_heads = 0, n_sets = 1, shape = 0, n_global = 0, rho_num = 1, rho_den = 4, tiling = 0;
   float sm_scale = 0.125f;
   int32_t kernel = LITEVAR_KERNEL_AUTO;
   int device = 0;

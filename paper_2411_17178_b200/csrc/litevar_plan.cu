@@ -72,28 +72,58 @@ __global__ void bounds_kernel(Schedule sc, int k0, const int32_t* radius_row, in
 }
 
 // ------------------------------------------------------------------ element predicate over one tile pair
-struct TileGeom {
+struct PlanGeom {
   int k0;           // 0-based step
   int s_k, n_k, L_k;
   int n_key_tiles;
   int shape;
+  int raster_len;             // cache rows covered by raster key tiles
+  const TileGeom* q_geom;     // [n_q_tiles]
+  const TileGeom* key_geom;   // [n_key_tiles]
 };
 
+// Query token (within the current scale) of slot m of a query tile, or -1 for a padding slot.
+__device__ __forceinline__ int query_slot_token(const TileGeom& g, int m, int s_k, int n_k, int& r, int& c) {
+  if (g.scale < 0) {
+    int q = g.a + m;
+    if (q >= n_k) return -1;
+    r = q / s_k;
+    c = q - r * s_k;
+    return q;
+  }
+  r = g.a + m / kPatchCols;
+  c = g.b + m % kPatchCols;
+  if (r >= s_k || c >= s_k) return -1;
+  return r * s_k + c;
+}
+
 // Live bits of query slot `m` of query tile `qt` against the 128 key slots of key tile `kt`.
-// Must be called by all 128 threads of the block (fills shared key-slot tables).
-__device__ uint4 tile_row_bits(const Schedule& sc, const TileGeom& g, const int2* __restrict__ bounds,
+// Must be called by all 128 threads of the block (fills shared key-slot tables).  `q_out` receives the
+// query token of the slot (-1: padding slot, all bits zero).
+__device__ uint4 tile_row_bits(const Schedule& sc, const PlanGeom& g, const int2* __restrict__ bounds,
                                const int32_t* __restrict__ radius_row, int qt, int kt,
-                               int16_t* ks_j, int16_t* ks_r, int16_t* ks_c, int32_t* ks_t) {
+                               int16_t* ks_j, int16_t* ks_r, int16_t* ks_c, int32_t* ks_t, int& q_out) {
   int m = threadIdx.x;
   {
-    int t = kt * kBlockN + m;  // raster key tiles: slot n of tile kt is cache row kt*128 + n
+    const TileGeom kg = g.key_geom[kt];
     int j = -1, r = 0, c = 0, tin = 0;
-    if (t < g.L_k) {
-      j = 0;
-      while (t >= sc.off[j + 1]) ++j;
-      tin = t - sc.off[j];
-      r = tin / sc.scale[j];
-      c = tin % sc.scale[j];
+    if (kg.scale < 0) {
+      int t = kg.a + m;  // raster key tile: slot n is cache row a + n, inside the raster prefix
+      if (t < g.raster_len) {
+        j = 0;
+        while (t >= sc.off[j + 1]) ++j;
+        tin = t - sc.off[j];
+        r = tin / sc.scale[j];
+        c = tin % sc.scale[j];
+      }
+    } else {
+      int s_j = sc.scale[kg.scale];
+      r = kg.a + m / kPatchCols;
+      c = kg.b + m % kPatchCols;
+      if (r < s_j && c < s_j) {
+        j = kg.scale;
+        tin = r * s_j + c;
+      }
     }
     ks_j[m] = (int16_t)j;
     ks_r[m] = (int16_t)r;
@@ -101,10 +131,11 @@ __device__ uint4 tile_row_bits(const Schedule& sc, const TileGeom& g, const int2
     ks_t[m] = tin;
   }
   __syncthreads();
-  int q = qt * kBlockM + m;
+  int r = 0, c = 0;
+  const int q = query_slot_token(g.q_geom[qt], m, g.s_k, g.n_k, r, c);
+  q_out = q;
   uint32_t w[4] = {0u, 0u, 0u, 0u};
-  if (q < g.n_k) {
-    int r = q / g.s_k, c = q % g.s_k;
+  if (q >= 0) {
     int cur_j = -2;
     int2 br = make_int2(0, -1), bc = make_int2(0, -1);
     long long band_ctr = 0;
@@ -141,15 +172,15 @@ __device__ uint4 tile_row_bits(const Schedule& sc, const TileGeom& g, const int2
 
 // ------------------------------------------------------------------ A3 pass 1: classify every candidate pair
 // cls: 0 dead, 1 partial, 2 full (every valid query slot sees all 128 key slots live).
-__global__ void __launch_bounds__(128) classify_kernel(Schedule sc, TileGeom g, const int2* bounds,
+__global__ void __launch_bounds__(128) classify_kernel(Schedule sc, PlanGeom g, const int2* bounds,
                                                        const int32_t* radius_row, uint8_t* cls,
                                                        int32_t* row_live, unsigned long long* live_entries) {
   __shared__ int16_t ks_j[kBlockN], ks_r[kBlockN], ks_c[kBlockN];
   __shared__ int32_t ks_t[kBlockN];
   int kt = blockIdx.x, qt = blockIdx.y;
-  uint4 b = tile_row_bits(sc, g, bounds, radius_row, qt, kt, ks_j, ks_r, ks_c, ks_t);
-  int q = qt * kBlockM + threadIdx.x;
-  bool valid = q < g.n_k;
+  int q;
+  uint4 b = tile_row_bits(sc, g, bounds, radius_row, qt, kt, ks_j, ks_r, ks_c, ks_t, q);
+  bool valid = q >= 0;
   int cnt = __popc(b.x) + __popc(b.y) + __popc(b.z) + __popc(b.w);
   int any = __syncthreads_or(cnt != 0);
   int all = __syncthreads_and(!valid || cnt == kBlockN);
@@ -214,7 +245,7 @@ __global__ void compact_kernel(int n_q_tiles, int n_key_tiles, const uint8_t* cl
 }
 
 // ------------------------------------------------------------------ A3 pass 4: element masks of partial pairs
-__global__ void __launch_bounds__(128) mask_bits_kernel(Schedule sc, TileGeom g, const int2* bounds,
+__global__ void __launch_bounds__(128) mask_bits_kernel(Schedule sc, PlanGeom g, const int2* bounds,
                                                         const int32_t* radius_row, const int32_t* mask_block_of,
                                                         uint4* mask) {
   __shared__ int16_t ks_j[kBlockN], ks_r[kBlockN], ks_c[kBlockN];
@@ -222,7 +253,8 @@ __global__ void __launch_bounds__(128) mask_bits_kernel(Schedule sc, TileGeom g,
   int kt = blockIdx.x, qt = blockIdx.y;
   int blk = mask_block_of[qt * g.n_key_tiles + kt];
   if (blk < 0) return;  // uniform per block
-  uint4 b = tile_row_bits(sc, g, bounds, radius_row, qt, kt, ks_j, ks_r, ks_c, ks_t);
+  int q;
+  uint4 b = tile_row_bits(sc, g, bounds, radius_row, qt, kt, ks_j, ks_r, ks_c, ks_t, q);
   mask[(size_t)blk * kBlockM + threadIdx.x] = b;
 }
 
@@ -232,19 +264,32 @@ __global__ void empty_row_kernel(int n_k, const int32_t* row_live, int32_t* flag
 }
 
 // ------------------------------------------------------------------ debug: dense mask from the tile plan
-__global__ void __launch_bounds__(128) materialize_kernel(SetDesc sd, int n_k, int L_k, uint32_t* dense) {
+__global__ void __launch_bounds__(128) materialize_kernel(SetDesc sd, Schedule sc, PlanGeom g, uint32_t* dense) {
   int qt = blockIdx.x, m = threadIdx.x;
-  int q = qt * kBlockM + m;
-  if (q >= n_k) return;
-  int words = (L_k + 31) / 32;
+  int r, c;
+  const int q = query_slot_token(g.q_geom[qt], m, g.s_k, g.n_k, r, c);
+  if (q < 0) return;
+  int words = (g.L_k + 31) / 32;
   for (int p = sd.row_ptr[qt]; p < sd.row_ptr[qt + 1]; ++p) {
     Pair pr = sd.pairs[p];
     uint4 b = pr.mask_block < 0 ? make_uint4(~0u, ~0u, ~0u, ~0u)
                                 : sd.mask[(size_t)pr.mask_block * kBlockM + m];
     uint32_t w[4] = {b.x, b.y, b.z, b.w};
-    int w0 = pr.key_tile * kMaskWordsPerRow;
-    for (int i = 0; i < 4; ++i)
-      if (w0 + i < words) dense[(size_t)q * words + w0 + i] = w[i];
+    const TileGeom kg = g.key_geom[pr.key_tile];
+    for (int n = 0; n < kBlockN; ++n) {
+      if (!((w[n >> 5] >> (n & 31)) & 1u)) continue;
+      int t;
+      if (kg.scale < 0) {
+        t = kg.a + n;
+        if (t >= g.raster_len) continue;
+      } else {
+        int s_j = sc.scale[kg.scale];
+        int kr = kg.a + n / kPatchCols, kc = kg.b + n % kPatchCols;
+        if (kr >= s_j || kc >= s_j) continue;
+        t = sc.off[kg.scale] + kr * s_j + kc;
+      }
+      dense[(size_t)q * words + (t >> 5)] |= 1u << (t & 31);  // row q belongs to this thread alone
+    }
   }
 }
 
@@ -291,7 +336,7 @@ litevar_status_t plan_step_set(litevar_plan* plan, int k0, int set, cudaStream_t
   if (s != LITEVAR_OK) return s;
   bounds_kernel<<<(unsigned)(((k0 + 1) * st.s_k + 255) / 256), 256, 0, stream>>>(sc, k0, d_radius_row, ss.d_bounds);
 
-  TileGeom g{k0, st.s_k, st.n_k, st.L_k, st.n_key_tiles, plan->shape};
+  PlanGeom g{k0, st.s_k, st.n_k, st.L_k, st.n_key_tiles, plan->shape, st.raster_len, st.d_q_geom, st.d_key_geom};
   Scratch tmp;
   uint8_t* d_cls = nullptr;
   int32_t *d_row_live = nullptr, *d_partial_base = nullptr, *d_totals = nullptr, *d_blk = nullptr;
@@ -377,6 +422,7 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
     if (scales[i] < 1 || scales[i] > kMaxScale) return LITEVAR_ERR_INVALID_ARG;
   if (window->shape != LITEVAR_WINDOW_SQUARE && window->shape != LITEVAR_WINDOW_BAND) return LITEVAR_ERR_INVALID_ARG;
   if (window->n_sets < 1 || window->n_sets > 64) return LITEVAR_ERR_INVALID_ARG;
+  if (window->tiling < LITEVAR_TILING_AUTO || window->tiling > LITEVAR_TILING_PATCH) return LITEVAR_ERR_INVALID_ARG;
   if (!window->radius && (window->rho_den <= 0 || window->rho_num < 0 || window->n_global_scales < 0))
     return LITEVAR_ERR_INVALID_ARG;
   if (!window->radius && window->n_sets != 1) return LITEVAR_ERR_INVALID_ARG;
@@ -401,6 +447,7 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
   plan->n_global = window->n_global_scales;
   plan->rho_num = window->rho_num;
   plan->rho_den = window->rho_den;
+  plan->tiling = window->tiling;
   plan->sm_scale = sm_scale > 0.f ? sm_scale : 0.125f;
   Schedule& sc = plan->sched;
   memset(&sc, 0, sizeof(sc));
@@ -453,8 +500,42 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
     st.s_k = sc.scale[k0];
     st.n_k = st.s_k * st.s_k;
     st.L_k = sc.off[k0 + 1];
-    st.n_q_tiles = (st.n_k + kBlockM - 1) / kBlockM;
-    st.n_key_tiles = (st.L_k + kBlockN - 1) / kBlockN;
+    // tile geometry of the step: raster tiles of 128 consecutive tokens, or 8x16 patches of a scale's grid
+    // where the grid is large enough for a 2-D window to leave whole patches dead
+    {
+      const int q_min = plan->tiling == LITEVAR_TILING_PATCH ? 1 : (plan->tiling == LITEVAR_TILING_RASTER ? 1 << 30 : 48);
+      const int key_min = plan->tiling == LITEVAR_TILING_PATCH ? 4 : (plan->tiling == LITEVAR_TILING_RASTER ? 1 << 30 : 32);
+      st.q_patch = st.s_k >= q_min;
+      st.first_patch = k0 + 1;
+      if (st.q_patch) {  // patch key tiles only together with patch query tiles
+        int first = 0;
+        while (first <= k0 && sc.scale[first] < key_min) ++first;
+        if (k0 + 1 - first > kMaxPatchScales) first = k0 + 1 - kMaxPatchScales;
+        st.first_patch = first;
+      }
+      st.raster_len = sc.off[st.first_patch];
+      st.n_raster_tiles = (st.raster_len + kBlockN - 1) / kBlockN;
+      if (st.q_patch) {
+        for (int r = 0; r < st.s_k; r += kPatchRows)
+          for (int c = 0; c < st.s_k; c += kPatchCols) st.q_geom.push_back(TileGeom{k0, r, c, 0});
+      } else {
+        for (int q0 = 0; q0 < st.n_k; q0 += kBlockM) st.q_geom.push_back(TileGeom{-1, q0, 0, 0});
+      }
+      for (int t0 = 0; t0 < st.raster_len; t0 += kBlockN) st.key_geom.push_back(TileGeom{-1, t0, 0, 0});
+      for (int j = st.first_patch; j <= k0; ++j)
+        for (int r = 0; r < sc.scale[j]; r += kPatchRows)
+          for (int c = 0; c < sc.scale[j]; c += kPatchCols)
+            st.key_geom.push_back(TileGeom{j, r, c, j - st.first_patch});
+      st.n_q_tiles = (int32_t)st.q_geom.size();
+      st.n_key_tiles = (int32_t)st.key_geom.size();
+      if ((s = dev_alloc(plan, &st.d_q_geom, st.q_geom.size())) != LITEVAR_OK) return fail(s);
+      if ((s = dev_alloc(plan, &st.d_key_geom, st.key_geom.size())) != LITEVAR_OK) return fail(s);
+      if (cudaMemcpyAsync(st.d_q_geom, st.q_geom.data(), sizeof(TileGeom) * st.q_geom.size(), cudaMemcpyHostToDevice,
+                          stream) != cudaSuccess ||
+          cudaMemcpyAsync(st.d_key_geom, st.key_geom.data(), sizeof(TileGeom) * st.key_geom.size(),
+                          cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return fail(LITEVAR_ERR_CUDA);
+    }
     st.share = share && share->share_step && share->share_step[k0] != 0;
     st.sets.resize(plan->n_sets);
     std::vector<SetDesc> descs(plan->n_sets);
@@ -495,6 +576,18 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   p.n_k = st.n_k;
   p.L_k = st.L_k;
   p.n_heads = plan->n_heads;
+  p.q_geom = st.d_q_geom;
+  p.key_geom = st.d_key_geom;
+  p.s_k = st.s_k;
+  p.q_patch = st.q_patch ? 1 : 0;
+  p.raster_len = st.raster_len;
+  p.first_patch = st.first_patch;
+  p.n_patch_scales = step_k - st.first_patch;
+  for (int i = 0; i < kMaxPatchScales; ++i) {
+    const int j = st.first_patch + i;
+    p.patch_scale[i] = j < step_k ? plan->sched.scale[j] : 0;
+    p.patch_off[i] = j < step_k ? plan->sched.off[j] : 0;
+  }
   p.batch_computed = st.share ? batch_pairs : 2 * batch_pairs;
   p.share_offset = st.share ? batch_pairs : 0;
   p.sm_scale = plan->sm_scale;
@@ -547,21 +640,24 @@ litevar_status_t litevar_plan_export_tiles(const litevar_plan_t* plan, int32_t s
   if (s != LITEVAR_OK) return s;
   const Step& st = plan->steps[step_k - 1];
   const StepSet& ss = st.sets[set];
-  if (q_tile_geom)
-    for (int i = 0; i < st.n_q_tiles; ++i) {
-      int first = i * kBlockM, slots = st.n_k - first < kBlockM ? st.n_k - first : kBlockM;
-      q_tile_geom[4 * i + 0] = first;
-      q_tile_geom[4 * i + 1] = slots;
-      q_tile_geom[4 * i + 2] = 0;
-      q_tile_geom[4 * i + 3] = slots;
+  auto put = [&](int32_t* out, const TileGeom& g, int side, int base, int limit) {
+    if (g.scale < 0) {  // raster: one row of up to 128 consecutive tokens
+      int valid = limit - g.a < kBlockM ? limit - g.a : kBlockM;
+      out[0] = g.a; out[1] = kBlockM; out[2] = 0; out[3] = 1; out[4] = valid;
+    } else {            // patch: kPatchRows x kPatchCols cells at (a, b), clipped to the grid
+      int vr = side - g.a < kPatchRows ? side - g.a : kPatchRows;
+      int vc = side - g.b < kPatchCols ? side - g.b : kPatchCols;
+      out[0] = base + g.a * side + g.b; out[1] = kPatchCols; out[2] = side; out[3] = vr; out[4] = vc;
     }
+  };
+  if (q_tile_geom)
+    for (int i = 0; i < st.n_q_tiles; ++i) put(q_tile_geom + 5 * i, st.q_geom[i], st.s_k, 0, st.n_k);
   if (key_tile_geom)
     for (int i = 0; i < st.n_key_tiles; ++i) {
-      int first = i * kBlockN, slots = st.L_k - first < kBlockN ? st.L_k - first : kBlockN;
-      key_tile_geom[4 * i + 0] = first;
-      key_tile_geom[4 * i + 1] = slots;
-      key_tile_geom[4 * i + 2] = 0;
-      key_tile_geom[4 * i + 3] = slots;
+      const TileGeom& g = st.key_geom[i];
+      const int side = g.scale < 0 ? 0 : plan->sched.scale[g.scale];
+      const int base = g.scale < 0 ? 0 : plan->sched.off[g.scale];
+      put(key_tile_geom + 5 * i, g, side, base, st.raster_len);
     }
   LV_CUDA(cudaDeviceSynchronize());
   if (row_ptr)
@@ -603,8 +699,8 @@ litevar_status_t litevar_plan_materialize_mask(const litevar_plan_t* plan, int32
   size_t words = (size_t)((st.L_k + 31) / 32);
   LV_CUDA(cudaMemsetAsync(dev_bits, 0, sizeof(uint32_t) * words * st.n_k, stream));
   SetDesc sd{ss.d_row_ptr, ss.d_pairs, ss.d_mask};
-  materialize_kernel<<<(unsigned)st.n_q_tiles, 128, 0, stream>>>(sd, st.n_k, st.L_k,
-                                                                   static_cast<uint32_t*>(dev_bits));
+  PlanGeom g{step_k - 1, st.s_k, st.n_k, st.L_k, st.n_key_tiles, plan->shape, st.raster_len, st.d_q_geom, st.d_key_geom};
+  materialize_kernel<<<(unsigned)st.n_q_tiles, 128, 0, stream>>>(sd, plan->sched, g, static_cast<uint32_t*>(dev_bits));
   LV_CUDA(cudaGetLastError());
   return LITEVAR_OK;
 }

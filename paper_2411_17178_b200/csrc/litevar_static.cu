@@ -262,6 +262,14 @@ extern "C" litevar_status_t litevar_attn_forward_static(
   p.n_k = a.n_k;
   p.L_k = a.L_k;
   p.n_heads = n_heads;
+  p.q_geom = nullptr;  // raster tiles
+  p.key_geom = nullptr;
+  p.s_k = a.s_k;
+  p.q_patch = 0;
+  p.raster_len = a.L_k;
+  p.first_patch = step_k;
+  p.n_patch_scales = 0;
+  for (int i = 0; i < kMaxPatchScales; ++i) p.patch_scale[i] = p.patch_off[i] = 0;
   p.batch_computed = share_cfg ? batch_pairs : 2 * batch_pairs;
   p.share_offset = share_cfg ? batch_pairs : 0;
   p.sm_scale = sm_scale > 0.f ? sm_scale : 0.125f;

@@ -16,12 +16,17 @@ KERNELS = [binding.KERNEL_SIMT, binding.KERNEL_TCGEN05]
 KNAME = {binding.KERNEL_SIMT: "simt", binding.KERNEL_TCGEN05: "tcgen05"}
 
 
+TILINGS = [binding.TILING_RASTER, binding.TILING_PATCH]
+TNAME = {binding.TILING_RASTER: "raster", binding.TILING_PATCH: "patch"}
+
+
+@pytest.mark.parametrize("tiling", TILINGS, ids=lambda t: TNAME[t])
 @pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
 @pytest.mark.parametrize("scales", [(1, 2, 3, 4), (1, 2, 3, 4, 5), (1, 2, 3, 4, 6, 9), (1, 2, 3, 4, 5, 6, 8, 10, 13)])
-def test_tiny_schedules_every_output(scales, kernel):
+def test_tiny_schedules_every_output(scales, kernel, tiling):
     lib_ready()
     w = wl.small_workload(scales, n_heads=3, batch_pairs=1)
-    plan = binding.Plan(scales, n_heads=3)
+    plan = binding.Plan(scales, n_heads=3, tiling=tiling)
     tab = orc.window_table(scales)
     Kc, Vc = wl.make_kv(w, 0)
     for k in w.steps:
@@ -49,12 +54,13 @@ def test_config1_full(kernel):
     plan.close()
 
 
+@pytest.mark.parametrize("tiling", TILINGS, ids=lambda t: TNAME[t])
 @pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
-def test_config2_one_layer_all_steps_with_sharing(kernel):
+def test_config2_one_layer_all_steps_with_sharing(kernel, tiling):
     lib_ready()
     w = wl.WORKLOADS[2]
     B = 2  # batch 2x2 here keeps the oracle fast; bench runs 2x8
-    plan = binding.Plan(w.scales, n_heads=w.n_heads, share_steps=[1] * 10)
+    plan = binding.Plan(w.scales, n_heads=w.n_heads, share_steps=[1] * 10, tiling=tiling)
     tab = orc.window_table(w.scales)
     Kc, Vc = wl.make_kv(w, 0, batch_rows=2 * B)
     for k in w.steps:
@@ -81,11 +87,12 @@ def _samples(rng, rows, H, n_k, count, s_k):
     return out
 
 
-def test_config4_final_steps_sampled():
+@pytest.mark.parametrize("tiling", [binding.TILING_AUTO, binding.TILING_PATCH], ids=["auto", "patch"])
+def test_config4_final_steps_sampled(tiling):
     lib_ready()
     w = wl.WORKLOADS[4]
     B = 1
-    plan = binding.Plan(w.scales, n_heads=w.n_heads, share_steps=[1] * 10)
+    plan = binding.Plan(w.scales, n_heads=w.n_heads, share_steps=[1] * 10, tiling=tiling)
     tab = orc.window_table(w.scales)
     Kc, Vc = wl.make_kv(w, 0, batch_rows=2 * B)
     rng = np.random.default_rng(4)
@@ -101,16 +108,17 @@ def test_config4_final_steps_sampled():
     plan.close()
 
 
+@pytest.mark.parametrize("tiling", [binding.TILING_AUTO, binding.TILING_RASTER], ids=["auto", "raster"])
 @pytest.mark.parametrize("rho", [(1, 8), (1, 4), (1, 2), None], ids=["rho1/8", "rho1/4", "rho1/2", "dense"])
-def test_config5_sampled(rho):
+def test_config5_sampled(rho, tiling):
     lib_ready()
     w = wl.WORKLOADS[5]
     if rho is None:
         tab = orc.full_table(w.scales)
-        plan = binding.Plan(w.scales, n_heads=w.n_heads, radius=tab)
+        plan = binding.Plan(w.scales, n_heads=w.n_heads, radius=tab, tiling=tiling)
     else:
         tab = orc.window_table(w.scales, rho=rho)
-        plan = binding.Plan(w.scales, n_heads=w.n_heads, rho=rho)
+        plan = binding.Plan(w.scales, n_heads=w.n_heads, rho=rho, tiling=tiling)
     Kc, Vc = wl.make_kv(w, 0)
     Q = wl.make_q(w, 0, 14)
     got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, binding.KERNEL_TCGEN05)
@@ -149,7 +157,7 @@ def test_strided_layout_and_custom_scale(kernel):
     scales = wl.SCALES_256[:9]
     H, B, k = 3, 1, 9
     w = wl.small_workload(scales, n_heads=H, batch_pairs=B, index=92)
-    plan = binding.Plan(scales, n_heads=H, sm_scale=0.2)
+    plan = binding.Plan(scales, n_heads=H, sm_scale=0.2, tiling=binding.TILING_PATCH)
     tab = orc.window_table(scales)
     Kc, Vc = wl.make_kv(w, 0)
     Q = wl.make_q(w, 0, k)

@@ -15,6 +15,17 @@ CASES = [
 ]
 
 
+def tile_tokens(geom):
+    """Token of every slot of every tile (-1 = padding slot), from the exported tile geometry."""
+    out = np.full((len(geom), 128), -1, np.int64)
+    for i, (first, cols, stride, vr, vc) in enumerate(geom):
+        m = np.arange(128)
+        r, c = m // cols, m % cols
+        ok = (r < vr) & (c < vc)
+        out[i, ok] = first + r[ok] * stride + c[ok]
+    return out
+
+
 def check_step(plan, scales, k, w_row):
     n_k, L_k = orc.map_shape(scales, k)
     ref = orc.mask(scales, k, w_row)
@@ -24,10 +35,11 @@ def check_step(plan, scales, k, w_row):
     st = plan.stats(k)
     assert st["live_entries"] == int(ref.sum())
     t = plan.export_tiles(k)
-    nq, nk = (n_k + 127) // 128, (L_k + 127) // 128
-    assert t["q_tile_geom"].shape == (nq, 4) and t["key_tile_geom"].shape == (nk, 4)
-    assert t["q_tile_geom"][:, 0].tolist() == [128 * i for i in range(nq)]
-    assert int(t["q_tile_geom"][:, 1].sum()) == n_k and int(t["key_tile_geom"][:, 1].sum()) == L_k
+    qtok, ktok = tile_tokens(t["q_tile_geom"]), tile_tokens(t["key_tile_geom"])
+    # the tiles partition the queries of the step and the keys of the cache prefix
+    assert sorted(qtok[qtok >= 0].tolist()) == list(range(n_k))
+    assert sorted(ktok[ktok >= 0].tolist()) == list(range(L_k))
+    nq, nk = len(qtok), len(ktok)
     rp = t["row_ptr"]
     assert rp[0] == 0 and rp[-1] == len(t["pair_key_tile"]) == st["live_tiles"]
     assert st["full_tiles"] + st["partial_tiles"] == st["live_tiles"]
@@ -35,21 +47,27 @@ def check_step(plan, scales, k, w_row):
     # the list is exactly the set of tile pairs with a live entry, in canonical order, and the
     # full flag marks exactly the pairs whose every (valid query, key slot) entry is live
     for qt in range(nq):
-        rows = ref[qt * 128:(qt + 1) * 128]
+        rows = ref[qtok[qt][qtok[qt] >= 0]]
         expect, full = [], []
         for kt in range(nk):
-            blk = rows[:, kt * 128:(kt + 1) * 128]
+            valid = ktok[kt] >= 0
+            blk = rows[:, ktok[kt][valid]]
             if blk.any():
                 expect.append(kt)
-                full.append(int(blk.all() and blk.shape[1] == 128))
+                full.append(int(blk.all() and valid.all()))
         assert t["pair_key_tile"][rp[qt]:rp[qt + 1]].tolist() == expect
         assert t["pair_is_full"][rp[qt]:rp[qt + 1]].tolist() == full
 
 
+TILINGS = [binding.TILING_RASTER, binding.TILING_PATCH, binding.TILING_AUTO]
+TNAME = {binding.TILING_RASTER: "raster", binding.TILING_PATCH: "patch", binding.TILING_AUTO: "auto"}
+
+
+@pytest.mark.parametrize("tiling", TILINGS, ids=lambda t: TNAME[t])
 @pytest.mark.parametrize("scales,rho", CASES)
-def test_planner_matches_oracle_mask(scales, rho):
+def test_planner_matches_oracle_mask(scales, rho, tiling):
     lib_ready()
-    plan = binding.Plan(scales, n_heads=2, rho=rho)
+    plan = binding.Plan(scales, n_heads=2, rho=rho, tiling=tiling)
     w = orc.window_table(scales, rho=rho)
     for k in range(1, len(scales) + 1):
         rad, bnd = plan.export_bounds(k)
@@ -68,11 +86,12 @@ def test_planner_matches_oracle_mask(scales, rho):
     plan.close()
 
 
+@pytest.mark.parametrize("tiling", [binding.TILING_RASTER, binding.TILING_AUTO], ids=lambda t: TNAME[t])
 @pytest.mark.parametrize("rho", [(1, 8), (1, 4), (1, 2)])
-def test_planner_2k_final_step(rho):
+def test_planner_2k_final_step(rho, tiling):
     lib_ready()
     scales = wl.SCALES_2K
-    plan = binding.Plan(scales, n_heads=1, rho=rho)
+    plan = binding.Plan(scales, n_heads=1, rho=rho, tiling=tiling)
     w = orc.window_table(scales, rho=rho)
     got = plan.materialize_mask(14)
     total = 0
@@ -81,6 +100,11 @@ def test_planner_2k_final_step(rho):
         assert np.array_equal(got[r0:r0 + 2048], ref)
         total += int(ref.sum())
     assert plan.stats(14)["live_entries"] == total
+    if tiling == binding.TILING_AUTO:
+        # patches of the large grids: fewer executed tile pairs than raster tiles for the same mask
+        raster = binding.Plan(scales, n_heads=1, rho=rho, tiling=binding.TILING_RASTER)
+        assert plan.stats(14)["live_tiles"] < raster.stats(14)["live_tiles"]
+        raster.close()
     plan.close()
 
 
@@ -88,7 +112,7 @@ def test_full_table_is_all_live_and_all_tiles_listed():
     lib_ready()
     scales = wl.SCALES_256
     K = len(scales)
-    plan = binding.Plan(scales, n_heads=1, radius=orc.full_table(scales))
+    plan = binding.Plan(scales, n_heads=1, radius=orc.full_table(scales), tiling=binding.TILING_RASTER)
     for k in range(1, K + 1):
         n_k, L_k = orc.map_shape(scales, k)
         assert plan.materialize_mask(k).all()
