@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) fwd_simt_kernel(FwdParams
     }
   }
   if (q >= p.n_k) return;  // padding slot (whole warp)
-  const SetDesc sd = p.sets[p.head_to_set ? p.head_to_set[h] : 0];
+  const SetDesc sd = p.head_to_set ? p.sets[p.head_to_set[h]] : p.set0;
 
   const uint16_t* qrow = p.q + b * p.q_sb + h * p.q_sh + (int64_t)q * p.q_st;
   q_sh[warp][lane] = bf16_bits_to_float(qrow[lane]);

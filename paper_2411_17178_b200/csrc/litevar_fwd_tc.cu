@@ -152,22 +152,10 @@ __device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, i
       ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar))
       : "memory");
 }
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* src, int c0, int c1, int c2, int c3) {
-  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
-               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-               : "memory");
-}
-__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, const void* src, int c0, int c1, int c2, int c3,
-                                             int c4) {
-  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
-               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-               : "memory");
-}
-
-// Tensor maps of one launch.  q and o are rank 4 (raster query tiles) or rank 5 (patch query tiles); kr/vr
+// Tensor maps of one launch.  q is rank 4 (raster query tiles) or rank 5 (patch query tiles); kr/vr
 // cover the raster prefix of the cache; k2/v2[i] cover the grid of the i-th key scale tiled in patches.
 struct TensorMaps {
-  CUtensorMap q, o, kr, vr;
+  CUtensorMap q, kr, vr;
   CUtensorMap k2[kMaxPatchScales], v2[kMaxPatchScales];
 };
 
@@ -338,50 +326,45 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  __syncthreads();  // barriers initialised; the producer warp goes ahead, the others finish the set-up
+  if (threadIdx.x == 0) {  // Q of both halves: needs nothing from the plan
+    mbar_expect_tx(&sm.q_full, has1 ? 2 * kTileBytes : kTileBytes);
+    load_q_tile(sm.q[0], tm, p, qt0, h, b, &sm.q_full);
+    if (has1) load_q_tile(sm.q[1], tm, p, qt1, h, b, &sm.q_full);
+  }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  {  // the ones block; made visible to the tensor pipe (async proxy) before the barrier below
+  if (warp != 0) {  // the ones block; made visible to the tensor pipe (async proxy) before the barrier below
     uint4* o4 = reinterpret_cast<uint4*>(sm.ones);
-    for (int i = threadIdx.x; i < (int)(kTileBytes / 16); i += kThreads)
+    for (int i = threadIdx.x - 32; i < (int)(kTileBytes / 16); i += kThreads - 32)
       o4[i] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   // plan lookups (independent of the set-up above)
-  const SetDesc sd = p.sets[p.head_to_set ? p.head_to_set[h] : 0];
+  const SetDesc sd = p.head_to_set ? p.sets[p.head_to_set[h]] : p.set0;
   const int beg0 = __ldg(&sd.row_ptr[qt0]), end0 = __ldg(&sd.row_ptr[qt0 + 1]);
   const int beg1 = end0, end1 = has1 ? __ldg(&sd.row_ptr[qt1 + 1]) : end0;
-  // The producer lane (it initialised the barriers itself) starts the first copies before the set-up
-  // barrier: Q of both halves, K and V of the first listed key tile.
-  UnionWalk pw;
-  int p_issued = 0;
-  if (threadIdx.x == 0 && end1 > beg0) {
-    const bool ld0 = end0 > beg0, ld1 = end1 > beg1;
-    mbar_expect_tx(&sm.q_full, (ld0 ? kTileBytes : 0u) + (ld1 ? kTileBytes : 0u));
-    if (ld0) load_q_tile(sm.q[0], tm, p, qt0, h, b, &sm.q_full);
-    if (ld1) load_q_tile(sm.q[1], tm, p, qt1, h, b, &sm.q_full);
-    pw.init(sd.pairs, beg0, end0, beg1, end1);
-    bool l0, l1;
-    const int kt = pw.next(l0, l1);
-    mbar_expect_tx(&sm.k_full[0], kTileBytes);
-    load_kv_tile(sm.k[0], &tm.kr, tm.k2, p, kt, h, b, &sm.k_full[0]);
-    mbar_expect_tx(&sm.v_full[0], kTileBytes);
-    load_kv_tile(sm.v[0], &tm.vr, tm.v2, p, kt, h, b, &sm.v_full[0]);
-    p_issued = 1;
-  }
   tc_fence_before();
-  __syncthreads();
+  if (warp != 0) asm volatile("bar.sync 1, %0;" ::"n"(kThreads - 32) : "memory");  // TMEM address, ones block
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
   if (warp < 4) {
-    if (warp == 0 && lane == 0 && end1 > beg0) {
+    if (warp == 0 && lane == 0 && end1 <= beg0) {
+      // nothing listed for this CTA: only the Q copies are in flight; wait for them (bounded) before leaving
+      const unsigned long long ts = global_ns();
+      while (!mbar_try(&sm.q_full, 0u))
+        if (global_ns() - ts > kWaitLimitNs) break;
+    } else if (warp == 0 && lane == 0) {
       // ---------------------------------------------------------------- TMA producer
-      int issued = p_issued;
-      for (int i = p_issued; pw.has(); ++i) {
+      UnionWalk pw;
+      pw.init(sd.pairs, beg0, end0, beg1, end1);
+      int issued = 0;
+      for (int i = 0; pw.has(); ++i) {
         bool l0, l1;
         const int kt = pw.next(l0, l1);
         const int s = i % kStages, n = i / kStages;
@@ -594,45 +577,37 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       // the last PV product of this half (all earlier ones are complete by issue order)
       if (ok && (ok = mbar_wait(&sm.o_full[hh], (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status))) {
         tc_fence_after();
-        // normalised bf16 row into the half's Q buffer (its last reader, S_hh of the last tile, is done),
-        // in the 128-byte swizzle the output tensor map expects; one lane then stores the whole tile
+        // token of this thread's query slot (-1: padding slot)
+        int q = qt * kBlockM + m;
+        if (p.q_geom != nullptr) {
+          const TileGeom g = p.q_geom[qt];
+          if (g.scale < 0) {
+            q = g.a + m;
+          } else {
+            const int qr = g.a + m / kPatchCols, qc = g.b + m % kPatchCols;
+            q = (qr < p.s_k && qc < p.s_k) ? qr * p.s_k + qc : -1;
+          }
+        }
+        // this thread stores output columns [32 sub, 32 sub + 32) of its row
+        uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st + 32 * sub;
+        uint16_t* orow2 = orow + (int64_t)p.share_offset * p.o_sb;
         uint32_t l16[16];
         tmem_ld16(tO + kHeadDim, l16);  // row sum of the bf16 probabilities, from the ones block
         uint32_t r[32];
         tmem_ld32(tO + 32 * sub, r);
         tmem_wait_ld();
         const float inv = 1.f / __uint_as_float(l16[0]);
-        uint8_t* srow = sm.q[hh] + m * 128;
+        if (q >= 0 && q < p.n_k) {
 #pragma unroll
-        for (int e = 0; e < 32; e += 8) {
-          uint4 o4;
-          o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
-          o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-          o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-          o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-          const int chunk = 4 * sub + (e >> 3);
-          *reinterpret_cast<uint4*>(srow + ((chunk ^ (m & 7)) << 4)) = o4;
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.x_full[hh]);
-        if (warp == 4 + 8 * hh && lane == 0 &&
-            mbar_wait(&sm.x_full[hh], (uint32_t)(n_tiles & 1), abort_flag, p.status)) {
-          const int nb = p.share_offset > 0 ? 2 : 1;  // under CFG sharing the tile also goes to row b + B
-          for (int i = 0; i < nb; ++i) {
-            const int bo = b + i * p.share_offset;
-            if (p.q_geom == nullptr) {
-              tma_store_4d(&tm.o, sm.q[hh], 0, qt * kBlockM, h, bo);
-            } else {
-              const TileGeom g = p.q_geom[qt];
-              if (g.scale < 0)
-                tma_store_4d(&tm.o, sm.q[hh], 0, g.a, h, bo);
-              else
-                tma_store_5d(&tm.o, sm.q[hh], 0, g.b, g.a, h, bo);
-            }
+          for (int e = 0; e < 32; e += 8) {
+            uint4 o4;
+            o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
+            o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+            o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+            o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + e) = o4;
+            if (p.share_offset > 0) *reinterpret_cast<uint4*>(orow2 + e) = o4;
           }
-          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         }
       }
     }
@@ -719,14 +694,11 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
   if (attr_err != cudaSuccess) return LITEVAR_ERR_CUDA;
   TensorMaps tm;
   memset(&tm, 0, sizeof(tm));
-  const int64_t out_rows = p.batch_computed + p.share_offset;
   bool ok;
   if (p.q_patch)
-    ok = encode_patch(&tm.q, p.q, 0, p.s_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb) &&
-         encode_patch(&tm.o, p.out, 0, p.s_k, p.n_heads, out_rows, p.o_st, p.o_sh, p.o_sb);
+    ok = encode_patch(&tm.q, p.q, 0, p.s_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb);
   else
-    ok = encode_raster(&tm.q, p.q, p.n_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb) &&
-         encode_raster(&tm.o, p.out, p.n_k, p.n_heads, out_rows, p.o_st, p.o_sh, p.o_sb);
+    ok = encode_raster(&tm.q, p.q, p.n_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb);
   ok = ok && encode_raster(&tm.kr, p.k, p.raster_len, p.n_heads, p.batch_computed, p.k_st, p.k_sh, p.k_sb) &&
        encode_raster(&tm.vr, p.v, p.raster_len, p.n_heads, p.batch_computed, p.v_st, p.v_sh, p.v_sb);
   for (int i = 0; ok && i < p.n_patch_scales; ++i)

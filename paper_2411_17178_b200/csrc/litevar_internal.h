@@ -74,6 +74,7 @@ struct Step {
 struct FwdParams {
   const SetDesc* sets;          // [n_sets] for this step
   const int32_t* head_to_set;   // [H] or nullptr (all heads use set 0)
+  SetDesc set0;                 // copy of sets[0]: saves the kernels one dependent load when there is one set
   const uint16_t* q;
   const uint16_t* k;
   const uint16_t* v;

@@ -565,6 +565,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   FwdParams p;
   p.sets = st.d_sets;
   p.head_to_set = plan->n_sets > 1 ? plan->d_head_to_set : nullptr;
+  p.set0 = SetDesc{st.sets[0].d_row_ptr, st.sets[0].d_pairs, st.sets[0].d_mask};
   p.q = static_cast<const uint16_t*>(Q);
   p.k = static_cast<const uint16_t*>(Kc);
   p.v = static_cast<const uint16_t*>(Vc);
