@@ -160,6 +160,47 @@ def live_count(scales: Sequence[int], k: int, w_row: Sequence[int]) -> int:
     return int(mask(scales, k, w_row).sum())
 
 
+# ----------------------------------------------------------------------------- band window
+# Second reading of "window width w" around "the diagonal" of a part (Section 2, Fig. 2(a) caption):
+# taken literally in the flattened attention map, the diagonal of the [n_k, n_j] part joins its corners,
+# and the window is the band of key tokens within w of it.
+def band_centre(q: int, n_j: int, n_k: int) -> int:
+    """Key token of a part with n_j columns under the centre of query row q of n_k rows:
+    floor((q + 1/2) * n_j / n_k)."""
+    return ((2 * q + 1) * n_j) // (2 * n_k)
+
+
+def band_table(scales: Sequence[int], rho: Tuple[int, int] = (1, 7), n_global_scales: int = 3) -> np.ndarray:
+    """Half-widths b[k-1][j-1] = round-half-up(rho * n_j) in key tokens; GLOBAL for the first scales."""
+    K = len(scales)
+    w = np.full((K, K), GLOBAL, dtype=np.int64)
+    for k in range(1, K + 1):
+        for j in range(1, k + 1):
+            if j > n_global_scales:
+                w[k - 1, j - 1] = default_radius(int(scales[j - 1]) ** 2, rho[0], rho[1])
+    return w
+
+
+def mask_band(scales: Sequence[int], k: int, w_row: Sequence[int],
+              q_rows: Optional[Sequence[int]] = None) -> np.ndarray:
+    """Boolean live mask of step k under the band reading: key token t' of scale j is live for query q
+    iff |t' - band_centre(q)| <= w_row[j-1] (or the part is GLOBAL).  One comparison per pair."""
+    n_k, L_k = map_shape(scales, k)
+    off = offsets(scales)
+    q = np.arange(n_k, dtype=np.int64) if q_rows is None else np.asarray(q_rows, dtype=np.int64)
+    out = np.zeros((q.shape[0], L_k), dtype=bool)
+    for j in range(1, k + 1):
+        n_j = int(scales[j - 1]) ** 2
+        w = int(w_row[j - 1])
+        if w == GLOBAL:
+            out[:, off[j - 1]:off[j]] = True
+            continue
+        t = np.arange(n_j, dtype=np.int64)
+        ctr = ((2 * q + 1) * n_j) // (2 * n_k)
+        out[:, off[j - 1]:off[j]] = np.abs(t[None, :] - ctr[:, None]) <= w
+    return out
+
+
 def schedule_saving(scales: Sequence[int], w: np.ndarray) -> float:
     """Fraction of attention-map entries (hence of QK^T + PV FLOPs) removed over all steps."""
     dense = 0
@@ -198,12 +239,13 @@ def attention_rows(Qr: np.ndarray, K: np.ndarray, V: np.ndarray, live_rows: np.n
 
 def attention_step(scales: Sequence[int], k: int, w_row: Sequence[int], Q, Kc, Vc,
                    sm_scale: Optional[float] = None, share_cfg: bool = False,
-                   return_weights: bool = False):
+                   return_weights: bool = False, band: bool = False):
     """Step-k MDWA attention for the whole batch.
 
     Q [2B, H, n_k, d]; Kc, Vc [2B, H, >=L_k, d] (only the first L_k rows are read).
     With share_cfg (ASC, Section 3) rows b < B are computed and rows b + B are copies of
     them; the unconditional half of Q/K/V is never read.
+    `band` selects the band reading of the window (mask_band) instead of the square one.
     Returns out [2B, H, n_k, d] fp64 (and the weights [2B, H, n_k, L_k] if asked).
     """
     Qd, Kd, Vd = bf16_to_f64(Q), bf16_to_f64(Kc), bf16_to_f64(Vc)
@@ -212,7 +254,7 @@ def attention_step(scales: Sequence[int], k: int, w_row: Sequence[int], Q, Kc, V
     assert nq == n_k and Kd.shape[2] >= L_k and Vd.shape[2] >= L_k
     if sm_scale is None:
         sm_scale = 1.0 / np.sqrt(d)
-    lv = mask(scales, k, w_row)
+    lv = mask_band(scales, k, w_row) if band else mask(scales, k, w_row)
     out = np.empty((rows, H, n_k, d), dtype=np.float64)
     wts = np.empty((rows, H, n_k, L_k), dtype=np.float64) if return_weights else None
     if share_cfg:

@@ -235,3 +235,41 @@ def test_forward_argument_errors():
     assert plan.forward_raw(**args(q_str=(1024, 1024, 60))) == 1
     torch.cuda.synchronize()
     plan.close()
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_band_window_forward(kernel):
+    # band reading of the window: same kernels, another plan
+    lib_ready()
+    scales = wl.SCALES_256
+    H, B = 3, 1
+    w = wl.small_workload(scales, n_heads=H, batch_pairs=B, share_cfg=True, index=98)
+    plan = binding.Plan(scales, n_heads=H, shape=binding.WINDOW_BAND, rho=(1, 7), share_steps=[1] * len(scales))
+    tab = orc.band_table(scales)
+    Kc, Vc = wl.make_kv(w, 0)
+    for k in (5, 8, 10):
+        Q = wl.make_q(w, 0, k)
+        got, _ = run_forward(plan, k, B, Q, Kc, Vc, kernel)
+        ref = orc.attention_step(scales, k, tab[k - 1], Q, Kc, Vc, share_cfg=True, band=True)
+        assert_close(got, ref, f"band step {k}")
+    plan.close()
+
+
+def test_band_window_2k_sampled():
+    lib_ready()
+    w = wl.WORKLOADS[5]
+    tab = orc.band_table(w.scales)
+    plan = binding.Plan(w.scales, n_heads=w.n_heads, shape=binding.WINDOW_BAND, rho=(1, 7))
+    Kc, Vc = wl.make_kv(w, 0)
+    Q = wl.make_q(w, 0, 14)
+    got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, binding.KERNEL_TCGEN05)
+    rng = np.random.default_rng(6)
+    smp = _samples(rng, 2, w.n_heads, 16384, 128, 128)
+    lv = orc.mask_band(w.scales, 14, tab[13], q_rows=[q for _, _, q in smp])
+    L = orc.map_shape(w.scales, 14)[1]
+    ref = np.stack([orc.attention_rows(orc.bf16_to_f64(Q[b, h, q:q + 1]), orc.bf16_to_f64(Kc[b, h, :L]),
+                                       orc.bf16_to_f64(Vc[b, h, :L]), lv[i:i + 1], 0.125)[0]
+                    for i, (b, h, q) in enumerate(smp)])
+    g = np.stack([got[b, h, q] for b, h, q in smp])
+    assert_close(g, ref, "band 2K")
+    plan.close()

@@ -199,6 +199,86 @@ def test_literal_three_parts_variant():
     assert m[:, :55].all() and not m[:, 55:].all()
 
 
+# ---------------------------------------------------------------- band reading of the window
+def _band_live_rational(scales, k, w_row, q, t):
+    """Exact rationals: the part's column whose interval [t'/n_j, (t'+1)/n_j) holds the centre
+    (q + 1/2)/n_k of the query row is found by interval membership; live = within w columns of it."""
+    off = [0]
+    for s in scales:
+        off.append(off[-1] + s * s)
+    j = next(j for j in range(1, k + 1) if off[j - 1] <= t < off[j])
+    w = w_row[j - 1]
+    if w < 0:
+        return True
+    n_j, n_k = scales[j - 1] ** 2, scales[k - 1] ** 2
+    ctr = (Fraction(q) + Fraction(1, 2)) / n_k
+    hits = [i for i in range(n_j) if Fraction(i, n_j) <= ctr < Fraction(i + 1, n_j)]
+    assert len(hits) == 1
+    return abs((t - off[j - 1]) - hits[0]) <= w
+
+
+@pytest.mark.parametrize("scales", [(1, 2, 3, 4), (1, 2, 3, 4, 5), (1, 2, 3, 4, 6, 9), (2, 3, 5, 7, 4)])
+@pytest.mark.parametrize("rho", [(1, 14), (1, 7), (2, 7)])
+def test_band_mask_brute_force_rationals(scales, rho):
+    w = orc.band_table(scales, rho=rho)
+    for k in range(1, len(scales) + 1):
+        n_k, L_k = orc.map_shape(scales, k)
+        m = orc.mask_band(scales, k, w[k - 1])
+        for q in range(n_k):
+            for t in range(L_k):
+                assert bool(m[q, t]) == _band_live_rational(scales, k, list(w[k - 1]), q, t)
+
+
+def test_band_counts_closed_form_and_invariants():
+    for scales in (S256, S512):
+        K = len(scales)
+        tabs = [orc.band_table(scales, rho=r) for r in ((1, 14), (1, 7), (2, 7), (1, 1))]
+        for k in range(1, K + 1):
+            n_k, L_k = orc.map_shape(scales, k)
+            ms = [orc.mask_band(scales, k, t[k - 1]) for t in tabs]
+            for a, b in zip(ms[:-1], ms[1:]):
+                assert not (a & ~b).any()                      # nested in the width
+            assert ms[-1].all()                                # a band as wide as the part is full attention
+            m, w = ms[1], tabs[1][k - 1]
+            off = orc.offsets(scales)
+            total = 0
+            for j in range(1, k + 1):
+                n_j = scales[j - 1] ** 2
+                if w[j - 1] < 0:
+                    total += n_k * n_j
+                    continue
+                for q in range(n_k):                           # clipped band length, min/max form
+                    c = math.floor((q + 0.5) * n_j / n_k + 1e-12)
+                    total += min(n_j - 1, c + w[j - 1]) - max(0, c - w[j - 1]) + 1
+            assert int(m.sum()) == total
+            own = m[:, off[k - 1]:off[k]]                       # own-scale part: |t - q| <= w, symmetric
+            assert (own == own.T).all() and own.diagonal().all()
+
+
+def test_band_default_saving_close_to_table1():
+    # the band stand-in b_j = round(n_j / 7) removes about as much as Table 1's threshold 0.95 (70.34 %)
+    dense = kept = 0
+    w = orc.band_table(S256)
+    for k in range(1, 11):
+        n_k, L_k = orc.map_shape(S256, k)
+        dense += n_k * L_k
+        kept += int(orc.mask_band(S256, k, w[k - 1]).sum())
+    assert abs(100 * (1 - kept / dense) - 70.34) < 1.0
+
+
+def test_band_attention_equals_library_attention_with_bool_mask():
+    scales = (1, 2, 3, 4, 5, 6, 8)
+    k = 7
+    w = orc.band_table(scales)
+    n_k, L_k = orc.map_shape(scales, k)
+    Q, Kc, Vc = _rand((2, 2, n_k, 64), 30), _rand((2, 2, L_k, 64), 31), _rand((2, 2, L_k, 64), 32)
+    out = orc.attention_step(scales, k, w[k - 1], Q, Kc, Vc, band=True)
+    m = torch.tensor([[_band_live_rational(scales, k, list(w[k - 1]), q, t) for t in range(L_k)]
+                      for q in range(n_k)])
+    ref = torch.nn.functional.scaled_dot_product_attention(Q.double(), Kc.double(), Vc.double(), attn_mask=m).numpy()
+    assert np.abs(out - ref).max() < 1e-12
+
+
 # ---------------------------------------------------------------- savings (Table 1, abstract)
 def test_default_window_saving_close_to_table1():
     # Table 1, threshold 0.95: 70.34 % FLOPs saving.  The synthetic default (rho = 1/4,

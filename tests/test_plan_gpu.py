@@ -155,3 +155,20 @@ def test_plan_errors_on_device():
     with pytest.raises(binding.LitevarError) as e:
         binding.Plan((1, 2, 3), n_heads=2, radius=np.zeros((1, 3, 3)), n_sets=1, head_to_set=[0, 1])
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("tiling", TILINGS, ids=lambda t: TNAME[t])
+@pytest.mark.parametrize("scales,rho", [((1, 2, 3, 4, 6, 9), (1, 7)), (wl.SCALES_256, (1, 7)), (wl.SCALES_256, (1, 14)),
+                                        (wl.SCALES_512, (1, 7))])
+def test_band_window_planner_matches_oracle(scales, rho, tiling):
+    # the literal reading of "window width w about the diagonal" (band in the flattened map)
+    lib_ready()
+    plan = binding.Plan(scales, n_heads=1, shape=binding.WINDOW_BAND, rho=rho, tiling=tiling)
+    w = orc.band_table(scales, rho=rho)
+    for k in range(1, len(scales) + 1):
+        rad, _ = plan.export_bounds(k)
+        assert rad.tolist() == w[k - 1].tolist()
+        ref = orc.mask_band(scales, k, w[k - 1])
+        assert np.array_equal(plan.materialize_mask(k), ref)
+        assert plan.stats(k)["live_entries"] == int(ref.sum())
+    plan.close()
