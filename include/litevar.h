@@ -49,8 +49,9 @@ enum { LITEVAR_WINDOW_SQUARE = 0, LITEVAR_WINDOW_BAND = 1 };
 /* Tile geometry of the plan.  RASTER: every query and key tile is 128 consecutive tokens.  PATCH:
  * a query tile is an 8 x 16 patch of the current scale's grid and the keys of the larger scales
  * are tiled in 8 x 16 patches of their own grids (grid-aligned), so that a 2-D window leaves whole
- * tiles dead; the coarse scales in front stay raster.  AUTO picks PATCH for steps whose grid side is
- * at least 48 (key scales of side >= 32 in patches, at most 8 of them) and RASTER otherwise. */
+ * tiles dead; the coarse scales in front stay raster.  AUTO picks PATCH for SQUARE windows at steps
+ * whose grid side is at least 48 (key scales of side >= 32 in patches, at most 8 of them) and RASTER
+ * otherwise. */
 enum { LITEVAR_TILING_AUTO = 0, LITEVAR_TILING_RASTER = 1, LITEVAR_TILING_PATCH = 2 };
 
 /* Window specification (paper Section 2: one window width per part of the step-k map; the

@@ -55,7 +55,7 @@ struct SharedStorage {
   alignas(1024) uint8_t ones[kTileBytes];  // bf16 1.0 everywhere: second N block of the PV product's B operand
   alignas(8) uint64_t q_full;
   uint64_t k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
-  uint64_t s_full[2], p_full[2], o_full[2], x_full[2];
+  uint64_t s_full[2], p_full[2][2], o_full[2], x_full[2];  // p_full[h][part]: P of the first / last two chunks of each thread
   float xmax[2][2][2][kBlockM];  // [tile parity][half][key half][row]: partial row maxima of a tile
   uint32_t tmem_base;
   int abort_flag;
@@ -318,7 +318,8 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sm.s_full[i], 1);
-      mbar_init(&sm.p_full[i], 8);
+      mbar_init(&sm.p_full[i][0], 8);
+      mbar_init(&sm.p_full[i][1], 8);
       mbar_init(&sm.o_full[i], 1);
       mbar_init(&sm.x_full[i], 8);
     }
@@ -421,16 +422,28 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
           if (i > 0 && prev_live[hh]) {  // O_hh += P_hh [V | 1]; P_hh sits in S_hh's columns
-            if (!(ok = mbar_wait(&sm.p_full[hh], (uint32_t)(n_pv[hh] & 1), abort_flag, p.status))) break;
+            // P arrives in two parts: key groups {0,1,4,5} (first two chunks of both threads of a row), then {2,3,6,7}
+            if (!(ok = mbar_wait(&sm.p_full[hh][0], (uint32_t)(n_pv[hh] & 1), abort_flag, p.status))) break;
             if (!v_ready) {
               if (!(ok = mbar_wait(&sm.v_full[prev_stage], prev_phase, abort_flag, p.status))) break;
               v_ready = true;
             }
             tc_fence_after();
 #pragma unroll
-            for (int kk = 0; kk < kBlockN / 16; ++kk)  // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns per step, key half 1 starts at S column 64
-              mma_ts(tmem + kColO + kOutCols * hh, tmem + kColS + 128 * hh + 8 * kk + (kk >= 4 ? 32 : 0),
-                     v_desc + (uint64_t)(2048 >> 4) * kk, kIdescPV, (n_pv[hh] > 0 || kk > 0) ? 1u : 0u);
+            for (int part = 0; part < 2; ++part) {
+              if (part == 1) {
+                if (!(ok = mbar_wait(&sm.p_full[hh][1], (uint32_t)(n_pv[hh] & 1), abort_flag, p.status))) break;
+                tc_fence_after();
+              }
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns per step, key half 1 starts at S column 64
+                const int kk = 2 * part + (g & 1) + 4 * (g >> 1);
+                mma_ts(tmem + kColO + kOutCols * hh, tmem + kColS + 128 * hh + 8 * kk + (kk >= 4 ? 32 : 0),
+                       v_desc + (uint64_t)(2048 >> 4) * kk, kIdescPV, (n_pv[hh] > 0 || part > 0 || g > 0) ? 1u : 0u);
+              }
+            }
+            if (!ok) break;
             mma_commit(&sm.o_full[hh]);
             ++n_pv[hh];
           }
@@ -518,6 +531,9 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
             mx1 = max3(mx1, __uint_as_float(rc[e + 2]), __uint_as_float(rc[e + 3]));
           }
         }
+        // the scores of the second pass start travelling while the maxima are exchanged
+        if (any_mixed) tmem_wait_st();  // the masked scores are read back
+        tmem_ld16(tS, r[0]);
         // the two threads of a row exchange their maxima
         float tile_max = fmaxf(mx0, mx1);
         sm.xmax[j & 1][hh][sub][m] = tile_max;
@@ -544,10 +560,8 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
             tmem_st16(tO + col, o);
           }
         }
-        if (any_mixed) tmem_wait_st();  // the masked scores are read back below
         // ---- pass 2: probabilities against the reference; P (packed bf16) over this thread's first 32 columns
         const float msc = row_max == -INFINITY ? 0.f : row_max * sc;
-        tmem_ld16(tS, r[0]);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t* rc = r[c & 1];
@@ -566,11 +580,17 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
             for (int e = 0; e < 8; ++e) pk[e] = 0u;
           }
           tmem_st8(tS + 8 * c, pk);  // columns [8c, 8c+8) of this thread's 64: inside chunks already read
+          if (c == 1) {  // first half of P can enter the PV product while the rest is formed
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.p_full[hh][0]);
+          }
         }
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.p_full[hh]);
+        if (lane == 0) mbar_arrive(&sm.p_full[hh][1]);
         pr = pr_next;
         mk = mk_next;
       }

@@ -503,8 +503,10 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
     // tile geometry of the step: raster tiles of 128 consecutive tokens, or 8x16 patches of a scale's grid
     // where the grid is large enough for a 2-D window to leave whole patches dead
     {
-      const int q_min = plan->tiling == LITEVAR_TILING_PATCH ? 1 : (plan->tiling == LITEVAR_TILING_RASTER ? 1 << 30 : 48);
-      const int key_min = plan->tiling == LITEVAR_TILING_PATCH ? 4 : (plan->tiling == LITEVAR_TILING_RASTER ? 1 << 30 : 32);
+      // AUTO: patches pay off for 2-D (square) windows on large grids; a band in token order wants raster tiles
+      const bool auto_patch = plan->tiling == LITEVAR_TILING_AUTO && plan->shape == LITEVAR_WINDOW_SQUARE;
+      const int q_min = plan->tiling == LITEVAR_TILING_PATCH ? 1 : (auto_patch ? 48 : 1 << 30);
+      const int key_min = plan->tiling == LITEVAR_TILING_PATCH ? 4 : 32;
       st.q_patch = st.s_k >= q_min;
       st.first_patch = k0 + 1;
       if (st.q_patch) {  // patch key tiles only together with patch query tiles
