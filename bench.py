@@ -37,7 +37,7 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
-from paper_2411_17178_b200 import workloads as wl  # noqa: E402
+from paper_2411_17178_b200 import sharding, workloads as wl  # noqa: E402
 
 FLOP_PER_ENTRY = 4 * wl.HEAD_DIM          # QK^T and PV, multiply + add, per live (q, t)
 TILE_FLOP = FLOP_PER_ENTRY * 128 * 128    # one executed 128x128 tile pair
@@ -169,22 +169,22 @@ def device_randn_bf16(shape, seed, device):
 class Buffers:
     """Device tensors of `n_sets` layers of one workload (seeded, generated on the device)."""
 
-    def __init__(self, w: wl.Workload, n_sets: int, device):
+    def __init__(self, w: wl.Workload, n_sets: int, device, seed_offset: int = 0):
         rows = 2 * w.batch_pairs
         L = wl.cache_len(w.scales, max(w.steps))
         self.k, self.v, self.q, self.out = [], [], [], []
         for layer in range(n_sets):
-            k = device_randn_bf16((rows, w.n_heads, L, wl.HEAD_DIM), wl.seed_for(w.index, layer, 0, 1), device)
+            k = device_randn_bf16((rows, w.n_heads, L, wl.HEAD_DIM), wl.seed_for(w.index, layer, 0, 1) + seed_offset, device)
             if w.key_head_scale:
                 k = (k.float() * wl.head_scales(w.n_heads).to(device).view(1, -1, 1, 1)).to(torch.bfloat16)
             self.k.append(k)
-            self.v.append(device_randn_bf16((rows, w.n_heads, L, wl.HEAD_DIM), wl.seed_for(w.index, layer, 0, 2),
+            self.v.append(device_randn_bf16((rows, w.n_heads, L, wl.HEAD_DIM), wl.seed_for(w.index, layer, 0, 2) + seed_offset,
                                             device))
             qs, outs = {}, {}
             for step in w.steps:
                 n_k = w.scales[step - 1] ** 2
                 qs[step] = device_randn_bf16((rows, w.n_heads, n_k, wl.HEAD_DIM),
-                                             wl.seed_for(w.index, layer, step, 0), device)
+                                             wl.seed_for(w.index, layer, step, 0) + seed_offset, device)
                 outs[step] = torch.empty_like(qs[step])
             self.q.append(qs)
             self.out.append(outs)
@@ -384,7 +384,7 @@ def gpu_arm(args):
     counts = schedule_counts(plan, w)
     useful, executed, nbytes = per_layer_work(w, counts, w.share_cfg)
     n_sets, per_set = sets_needed(w)
-    bufs = Buffers(w, n_sets, device)
+    bufs = Buffers(w, n_sets, device, seed_offset=sharding.rank_seed(0, rank))
     repeat = max(w.n_layers, n_sets)
     calls = generation_calls(w, n_sets, repeat)
     scale = repeat / w.n_layers
@@ -398,21 +398,24 @@ def gpu_arm(args):
             torch.cuda.synchronize()
         sampler.stop()
     status = plan.poll()
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    # ---- end to end with host buffers, on every rank (the host links are shared by the ranks of a node)
+    e2e_ms = h2d = d2h = None
+    if not args.kernel_only:
+        e2e_ms, h2d, d2h = time_e2e(plan, w, max(1, min(args.steps, 5)), 1, device)
+    # the job is as slow as its slowest rank
+    red = sharding.max_over_ranks([ms, e2e_ms if e2e_ms is not None else 0.0], device=device)
+    ms = red[0]
+    if e2e_ms is not None:
+        e2e_ms = red[1]
     ms_step = ms / scale
     gen_useful = useful * w.n_layers
-    value = world * gen_useful / (ms_step * 1e-3) / 1e12
+    value = sharding.whole_job_rate(gen_useful, world, ms_step) / 1e12
     launches_per_step = len(calls)
-
+    if world > 1:
+        import torch.distributed as dist
+        barrier()
+        dist.destroy_process_group()
     if rank != 0:
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-            dist.destroy_process_group()
         return
 
     out = {
@@ -457,9 +460,7 @@ def gpu_arm(args):
     eager_ms = time_eager(plan, w, bufs, calls, max(2, min(args.steps, 10)), 1) / scale
     out["eager_us_per_generation"] = round(eager_ms * 1e3, 2)
 
-    # ---- end to end with host buffers
-    e2e_ms, h2d, d2h = time_e2e(plan, w, max(1, min(args.steps, 5)), 1, device)
-    out["e2e"] = {"value": round(gen_useful / (e2e_ms * 1e-3) / 1e12 * world, 4), "unit": UNIT,
+    out["e2e"] = {"value": round(sharding.whole_job_rate(gen_useful, world, e2e_ms) / 1e12, 4), "unit": UNIT,
                   "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 4)}
     plan.close()
     del bufs

@@ -303,8 +303,11 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
   SharedStorage& sm = *reinterpret_cast<SharedStorage*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.y, b = blockIdx.z;
-  const int qt0 = 2 * blockIdx.x, qt1 = qt0 + 1;
+  // 1-D grid, heaviest query-tile pairs first: all (head, batch row) units of a pair are neighbours
+  const int n_units = p.n_heads * p.batch_computed;
+  const int pair_rank = blockIdx.x / n_units, unit = blockIdx.x - pair_rank * n_units;
+  const int h = unit % p.n_heads, b = unit / p.n_heads;
+  const int qt0 = 2 * (p.order ? __ldg(&p.order[pair_rank]) : pair_rank), qt1 = qt0 + 1;
   const bool has1 = qt1 < n_q_tiles;
   volatile int* abort_flag = &sm.abort_flag;
 
@@ -727,7 +730,7 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
          encode_patch(&tm.v2[i], p.v, p.patch_off[i], p.patch_scale[i], p.n_heads, p.batch_computed, p.v_st, p.v_sh,
                       p.v_sb);
   if (!ok) return LITEVAR_ERR_INVALID_ARG;
-  dim3 grid((unsigned)((n_q_tiles + 1) / 2), (unsigned)p.n_heads, (unsigned)p.batch_computed);
+  dim3 grid((unsigned)((n_q_tiles + 1) / 2) * (unsigned)p.n_heads * (unsigned)p.batch_computed);
   fwd_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tm, p, n_q_tiles);
   if (cudaGetLastError() != cudaSuccess) return LITEVAR_ERR_CUDA;
   return LITEVAR_OK;

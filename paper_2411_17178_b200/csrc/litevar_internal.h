@@ -54,6 +54,7 @@ struct StepSet {
   Pair* d_pairs = nullptr;
   uint4* d_mask = nullptr;
   int2* d_bounds = nullptr;  // [k][s_k] {lo, hi} per key scale and query row/column (SQUARE)
+  int32_t* d_order = nullptr;  // [ceil(n_q_tiles / 2)] query-tile pairs, heaviest first
 };
 
 struct Step {
@@ -75,6 +76,7 @@ struct FwdParams {
   const SetDesc* sets;          // [n_sets] for this step
   const int32_t* head_to_set;   // [H] or nullptr (all heads use set 0)
   SetDesc set0;                 // copy of sets[0]: saves the kernels one dependent load when there is one set
+  const int32_t* order;         // launch order of the query-tile pairs (heaviest first), or nullptr: natural order
   const uint16_t* q;
   const uint16_t* k;
   const uint16_t* v;

@@ -258,6 +258,22 @@ __global__ void __launch_bounds__(128) mask_bits_kernel(Schedule sc, PlanGeom g,
   mask[(size_t)blk * kBlockM + threadIdx.x] = b;
 }
 
+// Launch order of the CTAs of the forward kernel (one CTA = query tiles 2u and 2u+1): heaviest first, so
+// that the light corner tiles fill the tail of the grid.  Rank sort, one thread per CTA.
+__global__ void launch_order_kernel(int n_q_tiles, const int32_t* row_ptr, int32_t* order) {
+  const int n = (n_q_tiles + 1) / 2;
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u >= n) return;
+  auto work = [&](int v) { return row_ptr[min(2 * v + 2, n_q_tiles)] - row_ptr[2 * v]; };
+  const int mine = work(u);
+  int rank = 0;
+  for (int v = 0; v < n; ++v) {
+    const int wv = work(v);
+    rank += (wv > mine) || (wv == mine && v < u);
+  }
+  order[rank] = u;
+}
+
 __global__ void empty_row_kernel(int n_k, const int32_t* row_live, int32_t* flag) {
   int q = blockIdx.x * blockDim.x + threadIdx.x;
   if (q < n_k && row_live[q] == 0) atomicExch(flag, 1);
@@ -379,6 +395,10 @@ litevar_status_t plan_step_set(litevar_plan* plan, int k0, int set, cudaStream_t
   compact_kernel<<<(unsigned)((st.n_q_tiles + 127) / 128), 128, 0, stream>>>(
       st.n_q_tiles, st.n_key_tiles, d_cls, ss.d_row_ptr, d_partial_base, ss.d_pairs, d_blk);
   mask_bits_kernel<<<grid2, 128, 0, stream>>>(sc, g, ss.d_bounds, d_radius_row, d_blk, ss.d_mask);
+  s = dev_alloc(plan, &ss.d_order, (size_t)(st.n_q_tiles + 1) / 2);
+  if (s != LITEVAR_OK) return s;
+  launch_order_kernel<<<(unsigned)(((st.n_q_tiles + 1) / 2 + 127) / 128), 128, 0, stream>>>(st.n_q_tiles, ss.d_row_ptr,
+                                                                                         ss.d_order);
   LV_CUDA(cudaGetLastError());
   LV_CUDA(cudaStreamSynchronize(stream));  // scratch is freed when `tmp` goes out of scope
   return LITEVAR_OK;
@@ -568,6 +588,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   p.sets = st.d_sets;
   p.head_to_set = plan->n_sets > 1 ? plan->d_head_to_set : nullptr;
   p.set0 = SetDesc{st.sets[0].d_row_ptr, st.sets[0].d_pairs, st.sets[0].d_mask};
+  p.order = st.sets[0].d_order;
   p.q = static_cast<const uint16_t*>(Q);
   p.k = static_cast<const uint16_t*>(Kc);
   p.v = static_cast<const uint16_t*>(Vc);

@@ -252,6 +252,7 @@ extern "C" litevar_status_t litevar_attn_forward_static(
   p.sets = &sp->set;
   p.head_to_set = nullptr;
   p.set0 = SetDesc{sp->row_ptr, sp->pairs, sp->mask};  // device addresses inside the fixed array
+  p.order = nullptr;
   p.q = static_cast<const uint16_t*>(Q);
   p.k = static_cast<const uint16_t*>(Kc);
   p.v = static_cast<const uint16_t*>(Vc);
