@@ -330,8 +330,13 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  // Programmatic dependent launch: the next kernel in the stream may start its own set-up while this grid
+  // drains; this grid's set-up above ran while the previous one drained.  Nothing written by an earlier
+  // kernel is read before the wait below (the plan is immutable, Q/K/V are read by the producer lane only).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __syncthreads();  // barriers initialised; the producer warp goes ahead, the others finish the set-up
   if (threadIdx.x == 0) {  // Q of both halves: needs nothing from the plan
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     mbar_expect_tx(&sm.q_full, has1 ? 2 * kTileBytes : kTileBytes);
     load_q_tile(sm.q[0], tm, p, qt0, h, b, &sm.q_full);
     if (has1) load_q_tile(sm.q[1], tm, p, qt1, h, b, &sm.q_full);
@@ -731,8 +736,20 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
                       p.v_sb);
   if (!ok) return LITEVAR_ERR_INVALID_ARG;
   dim3 grid((unsigned)((n_q_tiles + 1) / 2) * (unsigned)p.n_heads * (unsigned)p.batch_computed);
-  fwd_tc_kernel<<<grid, kThreads, smem_bytes, stream>>>(tm, p, n_q_tiles);
-  if (cudaGetLastError() != cudaSuccess) return LITEVAR_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.overlap_launch ? 1 : 0;  // off when an earlier kernel of the stream writes what the set-up reads
+  if (cudaLaunchKernelEx(&cfg, fwd_tc_kernel, tm, p, n_q_tiles) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return LITEVAR_ERR_CUDA;
+  }
   return LITEVAR_OK;
 }
 

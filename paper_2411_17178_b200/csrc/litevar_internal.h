@@ -100,6 +100,8 @@ struct FwdParams {
   int32_t share_offset;         // B when the step is shared (second store at row b + B), else 0
   float sm_scale;
   int32_t* status;              // device word, set non-zero when a bounded wait expires
+  int32_t overlap_launch;       // 1: the tensor-core kernel may start its set-up before the previous kernel of the
+                                // stream has finished (the plan it reads was complete long before)
 };
 
 cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t stream);

@@ -616,6 +616,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   p.share_offset = st.share ? batch_pairs : 0;
   p.sm_scale = plan->sm_scale;
   p.status = plan->d_status;
+  p.overlap_launch = 1;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (plan->kernel == LITEVAR_KERNEL_SIMT) {
     cudaError_t e = launch_forward_simt(p, st.n_q_tiles, stream);
