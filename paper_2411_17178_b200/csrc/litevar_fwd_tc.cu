@@ -38,18 +38,29 @@ namespace litevar {
 
 namespace {
 
-constexpr int kStages = 4;
-constexpr int kThreads = 640;
 constexpr uint32_t kTileBytes = kBlockN * kHeadDim * 2;  // 16 KB: 128 rows of 128 B
-constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256;  // + 128 / kOutCols per half; P_h overlays S_h
+constexpr uint32_t kColS = 0;                // S_h at 128 h; O_h behind the S blocks; P_h overlays S_h
 constexpr int kOutCols = kHeadDim + 16;      // V columns + the ones block (row sums)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr int kNoTile = 0x7fffffff;
 
+// Two builds of the kernel.  Full: two query tiles per CTA, four K/V stages, 640 threads, all 512 TMEM
+// columns, one CTA per SM.  Lite (steps with a single query tile): one query tile, two stages, 384
+// threads, 256 TMEM columns, small enough for two CTAs per SM, so that consecutive calls overlap on an SM.
+template <int NH>
+struct Cfg {
+  static constexpr int kHalves = NH;
+  static constexpr int kStages = NH == 2 ? 4 : 2;
+  static constexpr int kThreads = 128 + 256 * NH;
+  static constexpr uint32_t kTmemCols = 256 * NH;
+  static constexpr int kMinCtas = NH == 2 ? 1 : 2;
+};
+
+template <int NH>
 struct SharedStorage {
-  alignas(1024) uint8_t q[2][kTileBytes];
+  static constexpr int kStages = Cfg<NH>::kStages;
+  alignas(1024) uint8_t q[NH][kTileBytes];
   alignas(1024) uint8_t k[kStages][kTileBytes];
   alignas(1024) uint8_t v[kStages][kTileBytes];
   alignas(1024) uint8_t ones[kTileBytes];  // bf16 1.0 everywhere: second N block of the PV product's B operand
@@ -297,18 +308,23 @@ struct UnionWalk {
   }
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+template <int NH>
+__global__ void __launch_bounds__(Cfg<NH>::kThreads, Cfg<NH>::kMinCtas)
 fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ FwdParams p, int n_q_tiles) {
+  constexpr int kStages = Cfg<NH>::kStages;
+  constexpr int kThreads = Cfg<NH>::kThreads;
+  constexpr uint32_t kTmemCols = Cfg<NH>::kTmemCols;
   extern __shared__ uint8_t smem_raw[];
-  SharedStorage& sm = *reinterpret_cast<SharedStorage*>(
+  constexpr uint32_t kColO = 128 * NH;
+  SharedStorage<NH>& sm = *reinterpret_cast<SharedStorage<NH>*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // 1-D grid, heaviest query-tile pairs first: all (head, batch row) units of a pair are neighbours
   const int n_units = p.n_heads * p.batch_computed;
   const int pair_rank = blockIdx.x / n_units, unit = blockIdx.x - pair_rank * n_units;
   const int h = unit % p.n_heads, b = unit / p.n_heads;
-  const int qt0 = 2 * (p.order ? __ldg(&p.order[pair_rank]) : pair_rank), qt1 = qt0 + 1;
-  const bool has1 = qt1 < n_q_tiles;
+  const int qt0 = NH * (p.order ? __ldg(&p.order[pair_rank]) : pair_rank), qt1 = qt0 + 1;
+  const bool has1 = NH == 2 && qt1 < n_q_tiles;
   volatile int* abort_flag = &sm.abort_flag;
 
   if (threadIdx.x == 0) {
@@ -339,7 +355,7 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
     asm volatile("griddepcontrol.wait;" ::: "memory");
     mbar_expect_tx(&sm.q_full, has1 ? 2 * kTileBytes : kTileBytes);
     load_q_tile(sm.q[0], tm, p, qt0, h, b, &sm.q_full);
-    if (has1) load_q_tile(sm.q[1], tm, p, qt1, h, b, &sm.q_full);
+    if (has1) load_q_tile(sm.q[NH - 1], tm, p, qt1, h, b, &sm.q_full);
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
@@ -404,7 +420,7 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       }
     } else if (warp == 1 && lane == 0 && end1 > beg0) {
       // ---------------------------------------------------------------- MMA issuer
-      const uint64_t q_desc[2] = {make_desc(smem_u32(sm.q[0])), make_desc(smem_u32(sm.q[1]))};
+      const uint64_t q_desc[2] = {make_desc(smem_u32(sm.q[0])), make_desc(smem_u32(sm.q[NH - 1]))};
       UnionWalk w;
       w.init(sd.pairs, beg0, end0, beg1, end1);
       bool ok = mbar_wait(&sm.q_full, 0u, abort_flag, p.status);
@@ -710,16 +726,36 @@ bool encode_patch(CUtensorMap* tm, const void* base, int64_t first_token, int64_
   return r == CUDA_SUCCESS;
 }
 
+
+template <int NH>
+litevar_status_t launch_variant(const TensorMaps& tm, const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
+  static std::once_flag attr_once;
+  static cudaError_t attr_err = cudaSuccess;
+  constexpr int smem_bytes = (int)sizeof(SharedStorage<NH>) + 1024;
+  std::call_once(attr_once, [] {
+    attr_err = cudaFuncSetAttribute(fwd_tc_kernel<NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  });
+  if (attr_err != cudaSuccess) return LITEVAR_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((n_q_tiles + NH - 1) / NH) * (unsigned)p.n_heads * (unsigned)p.batch_computed);
+  cfg.blockDim = dim3(Cfg<NH>::kThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.overlap_launch ? 1 : 0;  // off when an earlier kernel of the stream writes what the set-up reads
+  if (cudaLaunchKernelEx(&cfg, fwd_tc_kernel<NH>, tm, p, n_q_tiles) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return LITEVAR_ERR_CUDA;
+  }
+  return LITEVAR_OK;
+}
+
 }  // namespace
 
 litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
-  static std::once_flag attr_once;
-  static cudaError_t attr_err = cudaSuccess;
-  constexpr int smem_bytes = (int)sizeof(SharedStorage) + 1024;
-  std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
-  });
-  if (attr_err != cudaSuccess) return LITEVAR_ERR_CUDA;
   TensorMaps tm;
   memset(&tm, 0, sizeof(tm));
   bool ok;
@@ -735,22 +771,12 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
          encode_patch(&tm.v2[i], p.v, p.patch_off[i], p.patch_scale[i], p.n_heads, p.batch_computed, p.v_st, p.v_sh,
                       p.v_sb);
   if (!ok) return LITEVAR_ERR_INVALID_ARG;
-  dim3 grid((unsigned)((n_q_tiles + 1) / 2) * (unsigned)p.n_heads * (unsigned)p.batch_computed);
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem_bytes;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = p.overlap_launch ? 1 : 0;  // off when an earlier kernel of the stream writes what the set-up reads
-  if (cudaLaunchKernelEx(&cfg, fwd_tc_kernel, tm, p, n_q_tiles) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return LITEVAR_ERR_CUDA;
-  }
-  return LITEVAR_OK;
+  // A step with a single query tile and more CTAs than SMs runs the small build: two CTAs share an SM and
+  // hide each other's set-up and drain.  With fewer CTAs than SMs sharing would only halve each CTA's SM.
+  int dev = 0, n_sm = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) (void)cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  const bool lite = n_q_tiles == 1 && (long long)p.n_heads * p.batch_computed > n_sm;
+  return lite ? launch_variant<1>(tm, p, n_q_tiles, stream) : launch_variant<2>(tm, p, n_q_tiles, stream);
 }
 
 }  // namespace litevar
