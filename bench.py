@@ -348,7 +348,14 @@ def measure_config(w: wl.Workload, variant: str, rho, steps, warmup, device, pk,
                useful_frac_of_bf16_peak=round(useful * w.n_layers / (us_gen * 1e-6) / 1e12 / pk["bf16"], 4),
                hbm_gbs_compulsory=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9, 1),
                hbm_frac=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9 / pk["hbm"], 4),
-               buffer_sets=n_sets)
+               buffer_sets=n_sets, tiling="auto")
+    if len(w.steps) > 1:
+        # microseconds per call at every step: one graph of that step's calls over all layers
+        per_step = {}
+        for k in w.steps:
+            ms_k = time_graph(plan, w, bufs, [(k, layer % n_sets) for layer in range(repeat)], max(2, steps // 2), 2)
+            per_step[str(k)] = round(ms_k * 1e3 / repeat, 2)
+        res["us_per_call_by_step"] = per_step
     plan.close()
     return res, bufs
 

@@ -775,7 +775,10 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
   // hide each other's set-up and drain.  With fewer CTAs than SMs sharing would only halve each CTA's SM.
   int dev = 0, n_sm = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) (void)cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-  const bool lite = n_q_tiles == 1 && (long long)p.n_heads * p.batch_computed > n_sm;
+  const long long units = (long long)p.n_heads * p.batch_computed;
+  // ... and so does a step whose lists are short (set-up and drain weigh more than the shared K/V staging saves)
+  const bool lite = (n_q_tiles == 1 && units > n_sm) ||
+                    (units * n_q_tiles >= 2LL * n_sm && p.pairs_per_tile > 0 && p.pairs_per_tile <= 14);
   return lite ? launch_variant<1>(tm, p, n_q_tiles, stream) : launch_variant<2>(tm, p, n_q_tiles, stream);
 }
 

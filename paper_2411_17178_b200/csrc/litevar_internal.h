@@ -100,6 +100,7 @@ struct FwdParams {
   int32_t share_offset;         // B when the step is shared (second store at row b + B), else 0
   float sm_scale;
   int32_t* status;              // device word, set non-zero when a bounded wait expires
+  int32_t pairs_per_tile;       // average live key tiles per query tile (0: unknown); picks the kernel build
   int32_t overlap_launch;       // 1: the tensor-core kernel may start its set-up before the previous kernel of the
                                 // stream has finished (the plan it reads was complete long before)
 };

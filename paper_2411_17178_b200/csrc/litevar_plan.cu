@@ -617,6 +617,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   p.sm_scale = plan->sm_scale;
   p.status = plan->d_status;
   p.overlap_launch = 1;
+  p.pairs_per_tile = (st.sets[0].n_pairs + st.n_q_tiles - 1) / st.n_q_tiles;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (plan->kernel == LITEVAR_KERNEL_SIMT) {
     cudaError_t e = launch_forward_simt(p, st.n_q_tiles, stream);
