@@ -292,15 +292,31 @@ def time_e2e(plan, w: wl.Workload, steps, warmup, device):
         h2d += w.n_layers * comp * H * n_k * D * 2 * 3
         d2h += w.n_layers * rows * H * n_k * D * 2
 
+    # results travel back on a second stream, so a call's device-to-host copy overlaps the next call's
+    # host-to-device copies (the link is full duplex); two output buffers per step alternate
+    main, back = torch.cuda.current_stream(), torch.cuda.Stream()
+    do2 = {k: (do[k], torch.empty_like(do[k])) for k in w.steps}
+    freed = {k: [None, None] for k in w.steps}
+
     def generation():
         for k in w.steps:
             a, b = off[k - 1], off[k]
-            for _layer in range(w.n_layers):
+            for layer in range(w.n_layers):
+                i = layer & 1
+                if freed[k][i] is not None:
+                    main.wait_event(freed[k][i])
                 dq[k][:comp].copy_(host_q[k][:comp], non_blocking=True)
                 dk[:comp, :, a:b].copy_(new_k[k], non_blocking=True)
                 dv[:comp, :, a:b].copy_(new_v[k], non_blocking=True)
-                plan.forward(k, w.batch_pairs, dq[k], dk, dv, do[k])
-                host_out[k].copy_(do[k], non_blocking=True)
+                plan.forward(k, w.batch_pairs, dq[k], dk, dv, do2[k][i])
+                done = torch.cuda.Event()
+                done.record(main)
+                back.wait_event(done)
+                with torch.cuda.stream(back):
+                    host_out[k].copy_(do2[k][i], non_blocking=True)
+                    freed[k][i] = torch.cuda.Event()
+                    freed[k][i].record(back)
+        main.wait_stream(back)
 
     for _ in range(warmup):
         generation()
