@@ -273,3 +273,32 @@ def test_band_window_2k_sampled():
     g = np.stack([got[b, h, q] for b, h, q in smp])
     assert_close(g, ref, "band 2K")
     plan.close()
+
+
+@pytest.mark.parametrize("cfg,steps", [(2, (1, 4, 8, 10)), (3, (6, 10)), (4, (7, 10))], ids=["cfg2", "cfg3", "cfg4"])
+def test_bench_launch_configuration_sampled(cfg, steps):
+    # the batch, head count, sharing and kernel build that bench.py times for this workload; outputs are
+    # checked on sampled rows the oracle computes one by one
+    lib_ready()
+    w = wl.WORKLOADS[cfg]
+    B = w.batch_pairs
+    plan = binding.Plan(w.scales, n_heads=w.n_heads, share_steps=[1] * len(w.scales))
+    tab = orc.window_table(w.scales)
+    Kc, Vc = wl.make_kv(w, 0, max_step=max(steps))
+    kd, vd = Kc.cuda(), Vc.cuda()
+    rng = np.random.default_rng(cfg)
+    for k in steps:
+        Q = wl.make_q(w, 0, k)
+        out = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        plan.forward(k, B, Q.cuda(), kd, vd, out)
+        torch.cuda.synchronize()
+        assert plan.poll() == 0
+        n_k, s_k = w.scales[k - 1] ** 2, w.scales[k - 1]
+        smp = _samples(rng, 2 * B, w.n_heads, n_k, 2 * B * w.n_heads, s_k)[::max(1, (2 * B * w.n_heads) // 192)]
+        ref = orc.attention_sampled(w.scales, k, tab[k - 1], Q, Kc, Vc, smp, share_cfg=True)
+        got = out.double().cpu().numpy()
+        g = np.stack([got[b, h, q] for b, h, q in smp])
+        assert np.isfinite(got).all()
+        assert_close(g, ref, f"config {cfg} step {k}")
+        assert torch.equal(out[:B].view(torch.int16), out[B:].view(torch.int16))
+    plan.close()
