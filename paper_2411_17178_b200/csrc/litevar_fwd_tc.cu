@@ -323,7 +323,8 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
   const int n_units = p.n_heads * p.batch_computed;
   const int pair_rank = blockIdx.x / n_units, unit = blockIdx.x - pair_rank * n_units;
   const int h = unit % p.n_heads, b = unit / p.n_heads;
-  const int qt0 = NH * (p.order ? __ldg(&p.order[pair_rank]) : pair_rank), qt1 = qt0 + 1;
+  // the launch order lists query-tile PAIRS; the one-tile build takes the tiles in natural order
+  const int qt0 = NH == 2 ? 2 * (p.order ? __ldg(&p.order[pair_rank]) : pair_rank) : pair_rank, qt1 = qt0 + 1;
   const bool has1 = NH == 2 && qt1 < n_q_tiles;
   volatile int* abort_flag = &sm.abort_flag;
 
