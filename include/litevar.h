@@ -30,7 +30,7 @@ typedef struct litevar_plan litevar_plan_t; /* opaque; owns its device buffers *
 typedef enum {
   LITEVAR_OK = 0,
   LITEVAR_ERR_INVALID_ARG = 1,    /* NULL pointer, size or index out of range, misaligned tensor */
-  LITEVAR_ERR_UNSUPPORTED = 2,    /* valid request that this build does not implement */
+  LITEVAR_ERR_UNSUPPORTED = 2,    /* valid request that this library does not implement */
   LITEVAR_ERR_EMPTY_ROW = 3,      /* the window table leaves some query with no live key */
   LITEVAR_ERR_ARCH = 4,           /* current device is not compute capability 10.x */
   LITEVAR_ERR_OOM = 5,            /* device or host allocation failed */

@@ -1,6 +1,7 @@
 """CUDA forward path against the CPU oracle, through the C ABI, on the same seeded inputs.
 
-Tolerance (stated by the benchmark spec for bf16 inputs with fp32 accumulation): max-abs 1e-2, relative L2 5e-3.
+Tolerance for bf16 inputs with fp32 accumulation: max-abs 1e-2, relative L2 5e-3 (bf16 rounding of the
+probabilities and of the output gives a relative L2 error near 2e-3).
 """
 import numpy as np
 import pytest
