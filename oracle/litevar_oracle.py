@@ -212,6 +212,41 @@ def schedule_saving(scales: Sequence[int], w: np.ndarray) -> float:
     return 1.0 - kept / dense
 
 
+# ----------------------------------------------------------------------------- window calibration
+def window_ratio(scales: Sequence[int], k: int, j: int, w: int, maps: np.ndarray) -> float:
+    """R_w of part j of the step-k maps (Section 2): the sum of all attention values inside the window of
+    radius w divided by the sum of all values of the part.  maps: [n_maps, n_k, L_k], post-softmax."""
+    off = offsets(scales)
+    w_row = [GLOBAL] * len(scales)
+    w_row[j - 1] = w
+    inside = mask(scales, k, w_row)[:, off[j - 1]:off[j]]
+    part = np.asarray(maps, dtype=np.float64)[:, :, off[j - 1]:off[j]]
+    return float((part * inside[None]).sum() / part.sum())
+
+
+def calibrate_radius(scales: Sequence[int], k: int, maps: np.ndarray, r0: float,
+                     n_global_scales: int = 3) -> np.ndarray:
+    """Window design of Section 2, steps (1)-(3), for one step: for every part after the global ones the
+    window grows from zero until R_w reaches the threshold R_0; returns the radius row (GLOBAL for the
+    global parts and for unused entries j > k).  The decision is taken as inside >= R_0 * total in fp64."""
+    off = offsets(scales)
+    m = np.asarray(maps, dtype=np.float64)
+    out = np.full(len(scales), GLOBAL, dtype=np.int64)
+    for j in range(n_global_scales + 1, k + 1):
+        part = m[:, :, off[j - 1]:off[j]]
+        total = part.sum()
+        w = 0
+        while True:
+            w_row = [GLOBAL] * len(scales)
+            w_row[j - 1] = w
+            inside = (part * mask(scales, k, w_row)[None, :, off[j - 1]:off[j]]).sum()
+            if inside >= np.float64(np.float32(r0)) * total or w >= int(scales[j - 1]) - 1:
+                break
+            w += 1
+        out[j - 1] = w
+    return out
+
+
 # ----------------------------------------------------------------------------- attention
 def bf16_to_f64(x) -> np.ndarray:
     """Widen a torch bf16/fp32 tensor or numpy array to fp64 exactly."""

@@ -279,6 +279,71 @@ def test_band_attention_equals_library_attention_with_bool_mask():
     assert np.abs(out - ref).max() < 1e-12
 
 
+# ---------------------------------------------------------------- window calibration (Section 2, steps (1)-(3))
+def _dyadic_maps(scales, k, n_maps, seed):
+    """Non-negative maps on a grid of 1/1024: every partial sum is exact in fp64 in any order."""
+    rng = np.random.default_rng(seed)
+    n_k, L_k = orc.map_shape(scales, k)
+    return rng.integers(0, 64, size=(n_maps, n_k, L_k)).astype(np.float64) / 1024.0
+
+
+def test_calibration_uniform_maps_closed_form():
+    # uniform attention: R_w is the live fraction of the part, (sum of clipped 1-D window lengths)^2 / (n_k n_j)
+    scales, k = S256, 8
+    n_k, L_k = orc.map_shape(scales, k)
+    maps = np.ones((1, n_k, L_k))
+    s_k = scales[k - 1]
+    for j in (4, 6, 8):
+        s_j = scales[j - 1]
+        for w in (0, 1, 3):
+            A = sum(min(s_j - 1, math.floor((x + 0.5) * s_j / s_k + 1e-12) + w)
+                    - max(0, math.floor((x + 0.5) * s_j / s_k + 1e-12) - w) + 1 for x in range(s_k))
+            assert orc.window_ratio(scales, k, j, w, maps) == pytest.approx(A * A / (n_k * s_j * s_j), rel=1e-12)
+
+
+def test_calibration_recovers_a_planted_window():
+    # maps that are zero outside a window of radius w0 give exactly w0 at R_0 = 1, and less for a looser R_0
+    scales, k = S256[:9], 9
+    planted = [-1, -1, -1, 0, 1, 2, 2, 3, 4]
+    inside = orc.mask(scales, k, planted)
+    maps = _dyadic_maps(scales, k, 3, 1) + 1.0 / 1024
+    maps = maps * inside[None]
+    got = orc.calibrate_radius(scales, k, maps, 1.0)
+    assert got.tolist() == planted
+    loose = orc.calibrate_radius(scales, k, maps, 0.5)
+    assert all(a <= b for a, b in zip(loose.tolist(), planted)) and loose.tolist() != planted
+
+
+def test_calibration_monotone_and_limits():
+    scales, k = S256[:8], 8
+    maps = _dyadic_maps(scales, k, 2, 2) + 1.0 / 1024
+    prev = None
+    for r0 in (0.3, 0.6, 0.8, 0.95, 1.0):
+        rad = orc.calibrate_radius(scales, k, maps, r0)
+        assert rad[:3].tolist() == [-1, -1, -1]
+        if prev is not None:
+            assert (rad[3:k] >= prev[3:k]).all()              # a stricter threshold never shrinks a window
+        for j in range(4, k + 1):                             # smallest radius that reaches the threshold
+            w = int(rad[j - 1])
+            assert orc.window_ratio(scales, k, j, w, maps) >= np.float32(r0) - 1e-15
+            if w > 0:
+                assert orc.window_ratio(scales, k, j, w - 1, maps) < np.float32(r0)
+        prev = rad
+    # R_0 = 1 on strictly positive maps: full attention (Section 2), radius = the smallest that covers the part
+    full = orc.calibrate_radius(scales, k, maps, 1.0)
+    for j in range(4, k + 1):
+        w_row = [-1] * len(scales)
+        w_row[j - 1] = int(full[j - 1])
+        assert orc.mask(scales, k, w_row).all()
+    # all mass on the co-located key: radius 0
+    n_k, L_k = orc.map_shape(scales, k)
+    one_hot = np.zeros((1, n_k, L_k))
+    zero_row = [-1, -1, -1] + [0] * (k - 3)
+    one_hot[0][orc.mask(scales, k, zero_row)] = 1.0
+    one_hot[0][:, :14] = 0.0
+    assert orc.calibrate_radius(scales, k, one_hot, 1.0)[3:k].tolist() == [0] * (k - 3)
+
+
 # ---------------------------------------------------------------- savings (Table 1, abstract)
 def test_default_window_saving_close_to_table1():
     # Table 1, threshold 0.95: 70.34 % FLOPs saving.  The synthetic default (rho = 1/4,
