@@ -173,6 +173,25 @@ litevar_status_t litevar_attn_forward_static(const int32_t* scales, int32_t n_sc
                                              const void* Vcache, const litevar_strides_t* sv,
                                              void* out, const litevar_strides_t* so, void* stream);
 
+/*
+ * Window calibration of one step (paper Section 2, "detailed process of the MDWA pattern design", steps
+ * (1)-(3)): given saved post-softmax attention maps of step k, find for every part j after the global ones
+ * the smallest window radius w whose ratio R_w (sum of the map inside the window / sum of the whole part,
+ * taken over all given maps and query rows) reaches the threshold R_0.  Square windows only.
+ *
+ *   maps     device float32 [n_maps][n_k][L_k], contiguous, non-negative (rows need not sum to 1)
+ *   r0       threshold R_0 in (0, 1]; the decision is window mass >= (double)r0 * part mass in fp64
+ *   radius   host out [n_scales]: -1 for parts j <= n_global_scales and for j > step_k, else the radius;
+ *            a row of this kind is what litevar_window_t.radius takes
+ *   ratio    host out [n_scales][256] or NULL: R_w for w = 0 .. s_j - 1 (1 elsewhere)
+ *   stream   the kernel runs there; the call synchronises the stream and allocates 32 KB of scratch
+ * One pass over the maps (the kernel is bound by reading them once).
+ * Errors: INVALID_ARG, OOM, CUDA.
+ */
+litevar_status_t litevar_calibrate_windows(const int32_t* scales, int32_t n_scales, int32_t step_k,
+                                           int32_t n_global_scales, const float* maps, int64_t n_maps, float r0,
+                                           int32_t* radius, double* ratio, void* stream);
+
 /* Counts for step k and window set `set`: live map entries, live / full / partial tile pairs. */
 litevar_status_t litevar_plan_stats(const litevar_plan_t* plan, int32_t step_k, int32_t set,
                                     int64_t* live_entries, int64_t* live_tiles, int64_t* full_tiles,

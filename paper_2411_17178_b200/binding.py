@@ -24,7 +24,8 @@ KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
 TILING_AUTO, TILING_RASTER, TILING_PATCH = 0, 1, 2
 
 EXPORTS = (
-    "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_static", "litevar_plan_stats", "litevar_plan_tile_counts",
+    "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_static", "litevar_calibrate_windows",
+    "litevar_plan_stats", "litevar_plan_tile_counts",
     "litevar_plan_export_tiles", "litevar_plan_export_bounds", "litevar_plan_materialize_mask",
     "litevar_plan_poll_device_status", "litevar_plan_set_kernel", "litevar_plan_destroy",
     "litevar_status_string",
@@ -77,6 +78,8 @@ def load() -> ctypes.CDLL:
                                                 ctypes.POINTER(_Window), I32, I32, I32,
                                                 P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides),
                                                 P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides), P]
+    lib.litevar_calibrate_windows.restype = ctypes.c_int
+    lib.litevar_calibrate_windows.argtypes = [ctypes.POINTER(I32), I32, I32, I32, P, I64, ctypes.c_float, P, P, P]
     lib.litevar_plan_stats.restype = ctypes.c_int
     lib.litevar_plan_stats.argtypes = [P, I32, I32] + [ctypes.POINTER(I64)] * 4
     lib.litevar_plan_tile_counts.restype = ctypes.c_int
@@ -276,6 +279,22 @@ def forward_static(scales: Sequence[int], n_heads: int, step_k: int, batch_pairs
         raise LitevarError(st, "litevar_attn_forward_static (head_dim must be 64, one window set, and the step "
                                f"may have at most {STATIC_MAX_PAIRS} candidate tile pairs)")
     _check(st, "litevar_attn_forward_static")
+
+
+def calibrate_windows(scales: Sequence[int], step_k: int, maps, r0: float, n_global_scales: int = 3,
+                      want_ratio: bool = False, stream=None):
+    """litevar_calibrate_windows on a CUDA float32 tensor [n_maps, n_k, L_k]; returns the radius row
+    (numpy int32 [n_scales]) and, if asked, the R_w curves [n_scales, 256]."""
+    lib = load()
+    K = len(scales)
+    assert maps.is_cuda and maps.dtype.is_floating_point and maps.element_size() == 4 and maps.is_contiguous()
+    rad = np.zeros(K, np.int32)
+    ratio = np.zeros((K, 256), np.float64) if want_ratio else None
+    st = lib.litevar_calibrate_windows(_i32_array(scales), K, int(step_k), int(n_global_scales), maps.data_ptr(),
+                                       int(maps.shape[0]), float(r0), rad.ctypes.data,
+                                       ratio.ctypes.data if want_ratio else None, _stream_ptr(stream))
+    _check(st, "litevar_calibrate_windows")
+    return (rad, ratio) if want_ratio else rad
 
 
 def status_string(status: int) -> str:
