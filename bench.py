@@ -376,6 +376,37 @@ def measure_config(w: wl.Workload, variant: str, rho, steps, warmup, device, pk,
     return res, bufs
 
 
+def measure_calibration(device, pk):
+    """Window calibration (paper Section 2, steps (1)-(3)) on synthetic post-softmax maps: one pass over the
+    maps, reported against the HBM roofline (bytes = the maps read once).  Not part of the timed step."""
+    from paper_2411_17178_b200 import binding
+    rows = []
+    for name, scales, k, n_maps in (("256px step 10, 80 samples x 16 heads", wl.SCALES_256, 10, 1280),
+                                    ("512px step 10, 64 maps", wl.SCALES_512, 10, 64),
+                                    ("2K step 14, 1 map", wl.SCALES_2K, 14, 1)):
+        n_k, L = scales[k - 1] ** 2, wl.cache_len(scales, k)
+        g = torch.Generator(device=device)
+        g.manual_seed(7)
+        maps = torch.rand(n_maps, n_k, L, generator=g, device=device)
+        maps /= maps.sum(-1, keepdim=True)
+        for _ in range(3):
+            rad = binding.calibrate_windows(scales, k, maps, 0.95)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(5):
+            rad = binding.calibrate_windows(scales, k, maps, 0.95)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 5
+        nbytes = maps.numel() * 4
+        rows.append({"workload": name, "map_bytes": nbytes, "ms_per_call": round(ms, 3),
+                     "gbs": round(nbytes / ms / 1e6, 1), "hbm_frac": round(nbytes / ms / 1e6 / pk["hbm"], 4),
+                     "radius_at_r0_0.95": [int(x) for x in rad]})
+        del maps
+        torch.cuda.empty_cache()
+    return rows
+
+
 def gpu_arm(args):
     from paper_2411_17178_b200 import build as lvbuild
     rank = int(os.environ.get("RANK", "0"))
@@ -507,6 +538,7 @@ def gpu_arm(args):
             del shared_bufs
             torch.cuda.empty_cache()
         out["all_configs"] = table
+        out["calibration"] = measure_calibration(device, pk)
     print(json.dumps(out), flush=True)
 
 
