@@ -357,6 +357,12 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
     mbar_expect_tx(&sm.q_full, has1 ? 2 * kTileBytes : kTileBytes);
     load_q_tile(sm.q[0], tm, p, qt0, h, b, &sm.q_full);
     if (has1) load_q_tile(sm.q[NH - 1], tm, p, qt1, h, b, &sm.q_full);
+    if (p.first_tile_zero) {  // key tile 0 (cache rows [0,128), raster) heads every list: no look-up needed
+      mbar_expect_tx(&sm.k_full[0], kTileBytes);
+      tma_load_4d(sm.k[0], &tm.kr, 0, 0, h, b, &sm.k_full[0]);
+      mbar_expect_tx(&sm.v_full[0], kTileBytes);
+      tma_load_4d(sm.v[0], &tm.vr, 0, 0, h, b, &sm.v_full[0]);
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
@@ -390,7 +396,12 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       UnionWalk pw;
       pw.init(sd.pairs, beg0, end0, beg1, end1);
       int issued = 0;
-      for (int i = 0; pw.has(); ++i) {
+      if (p.first_tile_zero) {  // item 0 is already on its way
+        bool l0, l1;
+        (void)pw.next(l0, l1);
+        issued = 1;
+      }
+      for (int i = issued; pw.has(); ++i) {
         bool l0, l1;
         const int kt = pw.next(l0, l1);
         const int s = i % kStages, n = i / kStages;

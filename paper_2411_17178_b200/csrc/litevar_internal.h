@@ -54,6 +54,7 @@ struct StepSet {
   Pair* d_pairs = nullptr;
   uint4* d_mask = nullptr;
   int2* d_bounds = nullptr;  // [k][s_k] {lo, hi} per key scale and query row/column (SQUARE)
+  bool first_tile_zero = false;  // every query tile lists key tile 0 first
   int32_t* d_order = nullptr;  // [ceil(n_q_tiles / 2)] query-tile pairs, heaviest first
 };
 
@@ -101,6 +102,7 @@ struct FwdParams {
   float sm_scale;
   int32_t* status;              // device word, set non-zero when a bounded wait expires
   int32_t pairs_per_tile;       // average live key tiles per query tile (0: unknown); picks the kernel build
+  int32_t first_tile_zero;      // 1: every query tile's list starts with key tile 0 (its copies start at once)
   int32_t overlap_launch;       // 1: the tensor-core kernel may start its set-up before the previous kernel of the
                                 // stream has finished (the plan it reads was complete long before)
 };

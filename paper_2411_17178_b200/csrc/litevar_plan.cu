@@ -274,6 +274,16 @@ __global__ void launch_order_kernel(int n_q_tiles, const int32_t* row_ptr, int32
   order[rank] = u;
 }
 
+// Does every query tile list key tile 0 first?  (It does whenever the first cache rows stay live for every
+// query, as under any window of the paper: the coarsest scales are global.)  The forward kernel then starts
+// the copies of that tile before it has read anything of the plan.
+__global__ void first_tile_kernel(int n_q_tiles, const int32_t* row_ptr, const Pair* pairs, int32_t* not_zero) {
+  const int qt = blockIdx.x * blockDim.x + threadIdx.x;
+  if (qt >= n_q_tiles) return;
+  const int b = row_ptr[qt], e = row_ptr[qt + 1];
+  if (e == b || pairs[b].key_tile != 0) atomicExch(not_zero, 1);
+}
+
 __global__ void empty_row_kernel(int n_k, const int32_t* row_live, int32_t* flag) {
   int q = blockIdx.x * blockDim.x + threadIdx.x;
   if (q < n_k && row_live[q] == 0) atomicExch(flag, 1);
@@ -399,8 +409,14 @@ litevar_status_t plan_step_set(litevar_plan* plan, int k0, int set, cudaStream_t
   if (s != LITEVAR_OK) return s;
   launch_order_kernel<<<(unsigned)(((st.n_q_tiles + 1) / 2 + 127) / 128), 128, 0, stream>>>(st.n_q_tiles, ss.d_row_ptr,
                                                                                          ss.d_order);
+  LV_CUDA(cudaMemsetAsync(d_totals, 0, sizeof(int32_t), stream));
+  first_tile_kernel<<<(unsigned)((st.n_q_tiles + 127) / 128), 128, 0, stream>>>(st.n_q_tiles, ss.d_row_ptr, ss.d_pairs,
+                                                                                d_totals);
+  int32_t not_zero = 1;
+  LV_CUDA(cudaMemcpyAsync(&not_zero, d_totals, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
   LV_CUDA(cudaGetLastError());
   LV_CUDA(cudaStreamSynchronize(stream));  // scratch is freed when `tmp` goes out of scope
+  ss.first_tile_zero = not_zero == 0;
   return LITEVAR_OK;
 }
 
@@ -617,6 +633,8 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   p.sm_scale = plan->sm_scale;
   p.status = plan->d_status;
   p.overlap_launch = 1;
+  p.first_tile_zero = st.raster_len > 0 ? 1 : 0;  // key tile 0 must be the raster tile of cache rows [0, 128)
+  for (const StepSet& ss : st.sets) p.first_tile_zero &= ss.first_tile_zero ? 1 : 0;
   p.pairs_per_tile = (st.sets[0].n_pairs + st.n_q_tiles - 1) / st.n_q_tiles;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (plan->kernel == LITEVAR_KERNEL_SIMT) {
