@@ -633,36 +633,46 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       // the last PV product of this half (all earlier ones are complete by issue order)
       if (ok && (ok = mbar_wait(&sm.o_full[hh], (uint32_t)((n_tiles - 1) & 1), abort_flag, p.status))) {
         tc_fence_after();
-        // token of this thread's query slot (-1: padding slot)
-        int q = qt * kBlockM + m;
-        if (p.q_geom != nullptr) {
-          const TileGeom g = p.q_geom[qt];
-          if (g.scale < 0) {
-            q = g.a + m;
-          } else {
-            const int qr = g.a + m / kPatchCols, qc = g.b + m % kPatchCols;
-            q = (qr < p.s_k && qc < p.s_k) ? qr * p.s_k + qc : -1;
-          }
-        }
-        // this thread stores output columns [32 sub, 32 sub + 32) of its row
-        uint16_t* orow = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + (int64_t)q * p.o_st + 32 * sub;
-        uint16_t* orow2 = orow + (int64_t)p.share_offset * p.o_sb;
         uint32_t l16[16];
         tmem_ld16(tO + kHeadDim, l16);  // row sum of the bf16 probabilities, from the ones block
         uint32_t r[32];
-        tmem_ld32(tO + 32 * sub, r);
+        tmem_ld32(tO + 32 * sub, r);    // output columns [32 sub, 32 sub + 32) of this thread's row
         tmem_wait_ld();
         const float inv = 1.f / __uint_as_float(l16[0]);
-        if (q >= 0 && q < p.n_k) {
+        // The warp's 32 rows x 64 B pass through its own 2 KB slice of the half's Q buffer (its last reader,
+        // S_hh of the last tile, is done), so that four neighbouring lanes store one row's 64 contiguous
+        // bytes instead of 32 lanes touching 32 different rows.  Chunk position XOR (row / 2) keeps both
+        // the writes and the reads free of bank conflicts.  No other warp touches the slice.
+        uint8_t* slice = sm.q[hh < NH ? hh : 0] + (((warp - 4) & 7) << 11);
 #pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 o4;
-            o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
-            o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-            o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-            o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + e) = o4;
-            if (p.share_offset > 0) *reinterpret_cast<uint4*>(orow2 + e) = o4;
+        for (int e = 0; e < 32; e += 8) {
+          uint4 o4;
+          o4.x = pack_bf16(__uint_as_float(r[e + 0]) * inv, __uint_as_float(r[e + 1]) * inv);
+          o4.y = pack_bf16(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+          o4.z = pack_bf16(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
+          o4.w = pack_bf16(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
+          *reinterpret_cast<uint4*>(slice + lane * 64 + ((((e >> 3) ^ (lane >> 1)) & 3) << 4)) = o4;
+        }
+        __syncwarp();
+        TileGeom g = TileGeom{-1, qt * kBlockM, 0, 0};
+        if (p.q_geom != nullptr) g = p.q_geom[qt];
+        uint16_t* obase = p.out + (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + 32 * sub;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+          const int rl = it * 8 + (lane >> 2), ch = lane & 3;  // row of the warp's 32, 16-byte chunk of its 64 bytes
+          const int mm = lane_group * 32 + rl;                  // query slot of that row
+          int q;                                                // its token (-1: padding slot)
+          if (g.scale < 0) {
+            q = g.a + mm;
+          } else {
+            const int qr = g.a + mm / kPatchCols, qc = g.b + mm % kPatchCols;
+            q = (qr < p.s_k && qc < p.s_k) ? qr * p.s_k + qc : -1;
+          }
+          const uint4 o4 = *reinterpret_cast<const uint4*>(slice + rl * 64 + (((ch ^ (rl >> 1)) & 3) << 4));
+          if (q >= 0 && q < p.n_k) {
+            uint16_t* dst = obase + (int64_t)q * p.o_st + 8 * ch;
+            *reinterpret_cast<uint4*>(dst) = o4;
+            if (p.share_offset > 0) *reinterpret_cast<uint4*>(dst + (int64_t)p.share_offset * p.o_sb) = o4;
           }
         }
       }
