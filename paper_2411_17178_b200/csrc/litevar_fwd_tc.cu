@@ -44,6 +44,7 @@ constexpr int kOutCols = kHeadDim + 16;      // V columns + the ones block (row 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 constexpr int kNoTile = 0x7fffffff;
+constexpr uint32_t kSlotSpinLimit = 1u << 26;  // polls of a shared-memory word before a softmax thread gives up
 
 // Two builds of the kernel.  Full: two query tiles per CTA, four K/V stages, 640 threads, all 512 TMEM
 // columns, one CTA per SM.  Lite (steps with a single query tile): one query tile, two stages, 384
@@ -66,8 +67,8 @@ struct SharedStorage {
   alignas(1024) uint8_t ones[kTileBytes];  // bf16 1.0 everywhere: second N block of the PV product's B operand
   alignas(8) uint64_t q_full;
   uint64_t k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
-  uint64_t s_full[2], p_full[2][2], o_full[2], x_full[2];  // p_full[h][part]: P of the first / last two chunks of each thread
-  float xmax[2][2][2][kBlockM];  // [tile parity][half][key half][row]: partial row maxima of a tile
+  uint64_t s_full[2], p_full[2][2], o_full[2];  // p_full[h][part]: P of the first / last two chunks of each thread
+  unsigned long long xslot[2][2][2][kBlockM];  // [tile parity][half][key half][row]: {tile number + 1, partial row max}
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -341,7 +342,6 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       mbar_init(&sm.p_full[i][0], 8);
       mbar_init(&sm.p_full[i][1], 8);
       mbar_init(&sm.o_full[i], 1);
-      mbar_init(&sm.x_full[i], 8);
     }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -375,6 +375,9 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
     for (int i = threadIdx.x - 32; i < (int)(kTileBytes / 16); i += kThreads - 32)
       o4[i] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // the exchange words of the softmax threads start with a tag no tile uses
+    unsigned long long* xs = &sm.xslot[0][0][0][0];
+    for (int i = threadIdx.x - 32; i < 8 * kBlockM; i += kThreads - 32) xs[i] = 0ull;
   }
   // plan lookups (independent of the set-up above)
   const SetDesc sd = p.head_to_set ? p.sets[p.head_to_set[h]] : p.set0;
@@ -572,11 +575,28 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
         tmem_ld16(tS, r[0]);
         // the two threads of a row exchange their maxima
         float tile_max = fmaxf(mx0, mx1);
-        sm.xmax[j & 1][hh][sub][m] = tile_max;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.x_full[hh]);
-        if (!(ok = mbar_wait(&sm.x_full[hh], (uint32_t)(j & 1), abort_flag, p.status))) break;
-        tile_max = fmaxf(tile_max, sm.xmax[j & 1][hh][sub ^ 1][m]);
+        // (one 8-byte shared-memory word per thread and tile parity, tagged with the tile number: the partner
+        // polls it; it can be at most one tile ahead, so two parities suffice)
+        {
+          volatile unsigned long long* mine = &sm.xslot[j & 1][hh][sub][m];
+          volatile unsigned long long* theirs = &sm.xslot[j & 1][hh][sub ^ 1][m];
+          *mine = ((unsigned long long)(uint32_t)(j + 1) << 32) | __float_as_uint(tile_max);
+          unsigned long long got = *theirs;
+          for (uint32_t spin = 0; (uint32_t)(got >> 32) != (uint32_t)(j + 1); ++spin) {
+            if ((spin & 1023u) == 1023u && (*abort_flag || spin > kSlotSpinLimit)) {
+              *abort_flag = 1;
+              atomicExch(p.status, 1);
+              ok = false;
+              break;
+            }
+            got = *theirs;
+          }
+          if (!__all_sync(0xffffffffu, ok)) {
+            ok = false;
+            break;
+          }
+          tile_max = fmaxf(tile_max, __uint_as_float((uint32_t)got));
+        }
         // the reference max moves only when the tile exceeds it by more than the threshold
         float alpha = 1.f;
         if ((tile_max - row_max) * sc > kRescaleThreshold) {  // false for tile_max = -inf, true for row_max = -inf
