@@ -13,10 +13,16 @@
 //                (TMEM lane): warps 4..7 / 12..15 take the first 64 keys of the tile, warps 8..11 /
 //                16..19 the last 64.  Pass 1 over 16-key chunks: element mask (mixed chunks only, written
 //                back to TMEM) and the row max of the thread's keys; the two partial maxima meet through
-//                shared memory and one mbarrier phase per tile.  The row's reference max moves only when
-//                the tile exceeds it by more than 2^8; only then is the accumulator rescaled.  Pass 2:
+//                tagged shared-memory words that the partner polls.  The row's reference max moves only
+//                when the tile exceeds it by more than 2^8; only then is the accumulator rescaled.  Pass 2:
 //                exponentials against the reference, P as packed bf16 written over the first 32 of the
-//                thread's own 64 S columns.  Chunks without a live key for the whole warp are skipped.
+//                thread's own 64 S columns and handed to the PV product in two parts.  Chunks without a
+//                live key for the whole warp are skipped.  The epilogue passes the rows through a per-warp
+//                shared-memory slice so that four lanes store one row's 64 contiguous bytes.
+// Launch: 1-D grid, query-tile pairs heaviest first; programmatic stream serialization lets the set-up of a
+// call overlap the drain of the previous kernel; when every list starts with key tile 0 its copies start
+// before any plan look-up.  A small build (one query tile, two stages, 384 threads, 256 TMEM columns, two
+// CTAs per SM) serves steps with a single query tile or short lists.
 // Row sums come from the tensor pipe: the B operand of the PV product is V (64 columns) followed by a
 // block of ones (16 columns), so accumulator column 64 holds sum_t P[q,t] of the very bf16 weights the
 // output uses; no per-element add is issued.
