@@ -45,6 +45,38 @@ def test_calibration_matches_oracle(scales, k, peaked):
     plan.close()
 
 
+def test_calibration_many_rows_per_warp():
+    """More (map, query) rows than resident warps: batches of several rows, several batch waves, and query
+    indices that wrap around from one map to the next inside a batch."""
+    lib_ready()
+    scales, k = (1, 2, 3, 4, 5, 6), 6
+    maps = dyadic_maps(scales, k, 3001, 3, peaked=True)
+    dev = torch.tensor(maps, dtype=torch.float32, device="cuda")
+    for r0 in (0.6, 0.9):
+        rad, ratio = binding.calibrate_windows(scales, k, dev, r0, want_ratio=True)
+        assert rad.tolist() == orc.calibrate_radius(scales, k, maps, r0).tolist()
+        for j in range(4, k + 1):
+            for w in range(scales[j - 1]):
+                assert ratio[j - 1, w] == pytest.approx(orc.window_ratio(scales, k, j, w, maps), rel=1e-12, abs=1e-15)
+
+
+def test_calibration_wide_parts():
+    """Parts of more than 256 keys, one for each count of 32-column chunks per key row the kernel
+    specialises on (1, 2, 3, 4 and the general case), ahead of a small step."""
+    lib_ready()
+    scales, k = (1, 2, 3, 70, 100, 40, 150, 33, 17, 5), 10
+    maps = dyadic_maps(scales, k, 3, 21)
+    centre = orc.mask(scales, k, [-1, -1, -1] + [s // 5 for s in scales[3:]])
+    maps = maps + (32.0 / 1024) * centre[None]
+    dev = torch.tensor(maps, dtype=torch.float32, device="cuda")
+    for r0 in (0.3, 0.7):
+        rad, ratio = binding.calibrate_windows(scales, k, dev, r0, want_ratio=True)
+        assert rad.tolist() == orc.calibrate_radius(scales, k, maps, r0).tolist()
+        for j in range(4, k + 1):
+            for w in (0, 1, scales[j - 1] // 3, scales[j - 1] - 2, scales[j - 1] - 1):
+                assert ratio[j - 1, w] == pytest.approx(orc.window_ratio(scales, k, j, w, maps), rel=1e-12, abs=1e-15)
+
+
 def test_calibration_planted_window_and_global_variants():
     lib_ready()
     scales, k = wl.SCALES_256, 10
