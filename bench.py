@@ -57,20 +57,23 @@ def peaks():
 def kernel_source_hash():
     import hashlib
     h = hashlib.sha256()
-    for f in ("litevar_fwd_tc.cu", "litevar_plan.cu", "litevar_internal.h"):
+    for f in ("litevar_fwd_tc.cu", "litevar_fwd_small.cu", "litevar_plan.cu", "litevar_internal.h"):
         h.update(open(os.path.join(ROOT, "paper_2411_17178_b200", "csrc", f), "rb").read())
     return h.hexdigest()
 
 
-def recorded_traffic():
-    """DRAM bytes per launch of the forward kernel on workload 2 from the committed ncu summary, or None
+KERNEL_NAMES = {1: "fwd_simt_kernel", 2: "fwd_tc_kernel", 3: "fwd_small_kernel"}
+
+
+def recorded_traffic(kernel="fwd_tc_kernel"):
+    """DRAM bytes per launch of that forward kernel on workload 2 from the committed ncu summary, or None
     when the kernel sources have changed since those counters were taken."""
     path = os.path.join(ROOT, "profiles", "fwd_tc_workload2_traffic.txt")
     try:
         kv = dict(l.strip().split("=", 1) for l in open(path) if "=" in l and not l.startswith("#"))
         if kv.get("source_sha256") != kernel_source_hash():
             return None
-        return int(kv["bytes_per_launch"])
+        return int(kv["bytes_per_launch." + kernel])
     except Exception:
         return None
 
@@ -86,12 +89,12 @@ def schedule_counts(plan, w: wl.Workload):
     return out
 
 
-def per_layer_work(w: wl.Workload, counts, share: bool):
-    """Useful FLOP, executed FLOP and compulsory HBM bytes of one layer's calls."""
+def per_layer_work(w: wl.Workload, counts, share: bool, steps=None):
+    """Useful FLOP, executed FLOP and compulsory HBM bytes of one layer's calls (of the given steps)."""
     rows = 2 * w.batch_pairs
     computed = w.batch_pairs if share else rows
     useful = executed = nbytes = 0
-    for k in w.steps:
+    for k in (w.steps if steps is None else steps):
         c = counts[k]
         useful += c["live"] * FLOP_PER_ENTRY * computed * w.n_heads
         executed += c["tiles"] * TILE_FLOP * computed * w.n_heads
@@ -372,6 +375,7 @@ def measure_config(w: wl.Workload, variant: str, rho, steps, warmup, device, pk,
             ms_k = time_graph(plan, w, bufs, [(k, layer % n_sets) for layer in range(repeat)], max(2, steps // 2), 2)
             per_step[str(k)] = round(ms_k * 1e3 / repeat, 2)
         res["us_per_call_by_step"] = per_step
+        res["kernel_by_step"] = {str(k): KERNEL_NAMES[plan.step_kernel(k)] for k in w.steps}
     plan.close()
     return res, bufs
 
@@ -494,16 +498,38 @@ def gpu_arm(args):
     if sampler:
         out["clocks"] = sampler.summary()
 
-    # ---- roofline of the forward kernel on this workload (the only kernel in the timed region)
-    alg_bytes_launch = nbytes * w.n_layers / (len(w.steps) * w.n_layers)
-    avg_launch_s = ms_step * 1e-3 / (len(w.steps) * w.n_layers)
+    # ---- roofline of the dominant forward kernel on this workload.  AUTO runs two kernels (small steps /
+    # the rest); each group of steps is replayed as its own graph and timed with CUDA events, the kernel
+    # with the larger share of the generation is the one reported.
+    groups = {}
+    for k in w.steps:
+        groups.setdefault(KERNEL_NAMES[plan.step_kernel(k)], []).append(k)
+    timed = {}
+    for name, ks in groups.items():
+        g_calls = [(k, layer % n_sets) for k in ks for layer in range(repeat)]
+        g_ms = time_graph(plan, w, bufs, g_calls, max(3, args.steps // 2), 3) / scale
+        timed[name] = dict(steps=ks, launches=len(ks) * w.n_layers, us=g_ms * 1e3,
+                           bytes=per_layer_work(w, counts, w.share_cfg, ks)[2] * w.n_layers)
+    total_us = sum(t["us"] for t in timed.values())
+    dom = max(timed, key=lambda n: timed[n]["us"])
+    d = timed[dom]
+    alg_bytes_launch = d["bytes"] / d["launches"]
+    avg_launch_s = d["us"] * 1e-6 / d["launches"]
     achieved = alg_bytes_launch / avg_launch_s / 1e9
     out["roofline"] = {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm"], "unit": "GB/s",
                        "frac": round(achieved / pk["hbm"], 4),
-                       "traffic": recorded_traffic() if (w.index == 2 and variant == "window" and not args.rho) else None,
-                       "kernel": "fwd_tc_kernel", "peak_source": pk["source"],
+                       "traffic": recorded_traffic(dom) if (w.index == 2 and variant == "window" and not args.rho) else None,
+                       "kernel": dom, "peak_source": pk["source"], "steps": d["steps"],
+                       "launches_per_generation": d["launches"],
+                       "share_of_generation_time": round(d["us"] / total_us, 4),
                        "algorithmic_bytes_per_launch": round(alg_bytes_launch),
-                       "avg_launch_us": round(avg_launch_s * 1e6, 3)}
+                       "avg_launch_us": round(avg_launch_s * 1e6, 3),
+                       "other_kernels": [
+                           {"kernel": n, "steps": t["steps"], "launches_per_generation": t["launches"],
+                            "avg_launch_us": round(t["us"] / t["launches"], 3),
+                            "share_of_generation_time": round(t["us"] / total_us, 4),
+                            "hbm_frac": round(t["bytes"] / (t["us"] * 1e-6) / 1e9 / pk["hbm"], 4)}
+                           for n, t in timed.items() if n != dom]}
 
     if args.kernel_only:
         plan.close()

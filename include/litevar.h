@@ -81,9 +81,11 @@ typedef struct {
 
 /* Forward kernel selection (testing / measurement). */
 enum {
-  LITEVAR_KERNEL_AUTO = 0,   /* tensor-core kernel for every step */
-  LITEVAR_KERNEL_SIMT = 1,   /* plain CUDA-core kernel (slow; cross-check and bring-up) */
-  LITEVAR_KERNEL_TCGEN05 = 2 /* tcgen05/TMEM/TMA kernel */
+  LITEVAR_KERNEL_AUTO = 0,    /* per step: the small-step kernel where the step fits it, else the tcgen05 kernel */
+  LITEVAR_KERNEL_SIMT = 1,    /* plain CUDA-core kernel (slow; cross-check and bring-up) */
+  LITEVAR_KERNEL_TCGEN05 = 2, /* tcgen05/TMEM/TMA kernel for every step */
+  LITEVAR_KERNEL_SMALL = 3    /* reported by litevar_plan_step_kernel only: warp-level mma kernel for steps with one
+                                 query tile, at most two raster key tiles and little work */
 };
 
 /*
@@ -234,8 +236,13 @@ litevar_status_t litevar_plan_materialize_mask(const litevar_plan_t* plan, int32
  * with this plan gave up on a bounded wait since the last poll (the flag is then cleared). */
 litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan);
 
-/* Select the forward kernel (LITEVAR_KERNEL_*).  Not thread-safe against concurrent forwards. */
+/* Select the forward kernel (LITEVAR_KERNEL_AUTO, _SIMT or _TCGEN05).  Not thread-safe against concurrent
+ * forwards. */
 litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel);
+
+/* Which kernel litevar_attn_forward launches for step_k under the current selection: *kernel receives
+ * LITEVAR_KERNEL_SIMT, _TCGEN05 or _SMALL.  Host only; the paper has no counterpart (it gives no kernel design). */
+litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t* kernel);
 
 /* Frees the plan and its device buffers.  NULL is allowed. */
 void litevar_plan_destroy(litevar_plan_t* plan);

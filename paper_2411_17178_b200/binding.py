@@ -20,14 +20,14 @@ OK = 0
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "EMPTY_ROW", 4: "ARCH", 5: "OOM", 6: "CUDA",
                 7: "DEVICE_TIMEOUT"}
 WINDOW_SQUARE, WINDOW_BAND = 0, 1
-KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05 = 0, 1, 2
+KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_SMALL = 0, 1, 2, 3
 TILING_AUTO, TILING_RASTER, TILING_PATCH = 0, 1, 2
 
 EXPORTS = (
     "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_static", "litevar_calibrate_windows",
     "litevar_plan_stats", "litevar_plan_tile_counts",
     "litevar_plan_export_tiles", "litevar_plan_export_bounds", "litevar_plan_materialize_mask",
-    "litevar_plan_poll_device_status", "litevar_plan_set_kernel", "litevar_plan_destroy",
+    "litevar_plan_poll_device_status", "litevar_plan_set_kernel", "litevar_plan_step_kernel", "litevar_plan_destroy",
     "litevar_status_string",
 )
 
@@ -94,6 +94,8 @@ def load() -> ctypes.CDLL:
     lib.litevar_plan_poll_device_status.argtypes = [P]
     lib.litevar_plan_set_kernel.restype = ctypes.c_int
     lib.litevar_plan_set_kernel.argtypes = [P, I32]
+    lib.litevar_plan_step_kernel.restype = ctypes.c_int
+    lib.litevar_plan_step_kernel.argtypes = [P, I32, ctypes.POINTER(I32)]
     lib.litevar_plan_destroy.restype = None
     lib.litevar_plan_destroy.argtypes = [P]
     lib.litevar_status_string.restype = ctypes.c_char_p
@@ -246,6 +248,12 @@ class Plan:
 
     def set_kernel(self, kernel: int) -> None:
         _check(self._lib.litevar_plan_set_kernel(self._h, int(kernel)), "litevar_plan_set_kernel")
+
+    def step_kernel(self, step_k: int) -> int:
+        """KERNEL_SIMT, KERNEL_TCGEN05 or KERNEL_SMALL: what a forward of this step launches."""
+        out = ctypes.c_int32(0)
+        _check(self._lib.litevar_plan_step_kernel(self._h, int(step_k), ctypes.byref(out)), "litevar_plan_step_kernel")
+        return int(out.value)
 
 
 STATIC_MAX_PAIRS = 2048

@@ -40,6 +40,13 @@ struct TileGeom {
 constexpr int kPatchRows = 8, kPatchCols = 16;  // kPatchRows * kPatchCols == 128
 constexpr int kMaxPatchScales = 8;              // key scales that can be tiled in 2-D patches
 
+// The whole tile list of a step with one query tile and at most two key tiles, passed to the small-step
+// kernel by value (saves it two dependent global loads).
+struct SmallLists {
+  int32_t n;
+  Pair pr[2];
+};
+
 // Device-visible tile plan of one (step, window set).
 struct SetDesc {
   const int32_t* row_ptr;  // [n_q_tiles + 1]
@@ -56,6 +63,7 @@ struct StepSet {
   int2* d_bounds = nullptr;  // [k][s_k] {lo, hi} per key scale and query row/column (SQUARE)
   bool first_tile_zero = false;  // every query tile lists key tile 0 first
   int32_t* d_order = nullptr;  // [ceil(n_q_tiles / 2)] query-tile pairs, heaviest first
+  SmallLists small = {-1, {{0, 0}, {0, 0}}};  // host copy of the tile list of a small step (n < 0: not a small step)
 };
 
 struct Step {
@@ -108,6 +116,11 @@ struct FwdParams {
 };
 
 cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
+
+// Small steps (one query tile, at most two raster key tiles, little enough work): warp-level mma on a shared-memory copy of the
+// whole K/V prefix.  `lists` is set 0's tile list (per-head sets are looked up on the device).
+bool small_step_eligible(int n_q_tiles, int n_key_tiles, bool raster_only, int n_k, int L_k);
+cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, cudaStream_t stream);
 
 // Tensor-core path.  Returns LITEVAR_OK or an error status (tensor-map encoding can fail).
 litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream);

@@ -425,6 +425,17 @@ bool strides_ok(const litevar_strides_t* s) {
          (s->head % 8) == 0 && (s->token % 8) == 0;
 }
 
+// The kernel a forward of this step launches under the plan's current selection.
+int32_t step_kernel(const litevar_plan_t* plan, const Step& st) {
+  if (plan->kernel == LITEVAR_KERNEL_SIMT) return LITEVAR_KERNEL_SIMT;
+  if (plan->kernel == LITEVAR_KERNEL_AUTO) {
+    bool all_small = true;  // every window set of the step has a list the small-step kernel can take
+    for (const StepSet& ss : st.sets) all_small = all_small && ss.small.n > 0;
+    if (all_small) return LITEVAR_KERNEL_SMALL;
+  }
+  return LITEVAR_KERNEL_TCGEN05;
+}
+
 }  // namespace
 
 extern "C" {
@@ -580,6 +591,14 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
     for (int set = 0; set < plan->n_sets; ++set) {
       if ((s = plan_step_set(plan, k0, set, stream)) != LITEVAR_OK) return fail(s);
       descs[set] = SetDesc{st.sets[set].d_row_ptr, st.sets[set].d_pairs, st.sets[set].d_mask};
+      StepSet& ss = st.sets[set];
+      if (small_step_eligible(st.n_q_tiles, st.n_key_tiles, !st.q_patch && st.first_patch == k0 + 1, st.n_k, st.L_k) &&
+          ss.n_pairs >= 1 && ss.n_pairs <= 2) {
+        ss.small.n = ss.n_pairs;
+        if (cudaMemcpyAsync(ss.small.pr, ss.d_pairs, sizeof(Pair) * ss.n_pairs, cudaMemcpyDeviceToHost, stream) !=
+            cudaSuccess)
+          return fail(LITEVAR_ERR_CUDA);
+      }
     }
     if ((s = dev_alloc(plan, &st.d_sets, (size_t)plan->n_sets)) != LITEVAR_OK) return fail(s);
     if (cudaMemcpyAsync(st.d_sets, descs.data(), sizeof(SetDesc) * plan->n_sets, cudaMemcpyHostToDevice,
@@ -637,6 +656,13 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   for (const StepSet& ss : st.sets) p.first_tile_zero &= ss.first_tile_zero ? 1 : 0;
   p.pairs_per_tile = (st.sets[0].n_pairs + st.n_q_tiles - 1) / st.n_q_tiles;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (step_kernel(plan, st) == LITEVAR_KERNEL_SMALL) {
+    if (launch_forward_small(p, st.sets[0].small, stream) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return LITEVAR_ERR_CUDA;
+    }
+    return LITEVAR_OK;
+  }
   if (plan->kernel == LITEVAR_KERNEL_SIMT) {
     cudaError_t e = launch_forward_simt(p, st.n_q_tiles, stream);
     if (e != cudaSuccess) {
@@ -764,6 +790,12 @@ litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan) {
 litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel) {
   if (!plan || kernel < LITEVAR_KERNEL_AUTO || kernel > LITEVAR_KERNEL_TCGEN05) return LITEVAR_ERR_INVALID_ARG;
   plan->kernel = kernel;
+  return LITEVAR_OK;
+}
+
+litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t* kernel) {
+  if (!plan || !kernel || step_k < 1 || step_k > plan->sched.n_scales) return LITEVAR_ERR_INVALID_ARG;
+  *kernel = step_kernel(plan, plan->steps[step_k - 1]);
   return LITEVAR_OK;
 }
 

@@ -13,8 +13,9 @@ from tests.gpu_util import assert_close, lib_ready, run_forward
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [binding.KERNEL_SIMT, binding.KERNEL_TCGEN05]
-KNAME = {binding.KERNEL_SIMT: "simt", binding.KERNEL_TCGEN05: "tcgen05"}
+# AUTO is what callers get: the small-step kernel where a step fits it, the tcgen05 kernel elsewhere
+KERNELS = [binding.KERNEL_SIMT, binding.KERNEL_TCGEN05, binding.KERNEL_AUTO]
+KNAME = {binding.KERNEL_SIMT: "simt", binding.KERNEL_TCGEN05: "tcgen05", binding.KERNEL_AUTO: "auto"}
 
 
 TILINGS = [binding.TILING_RASTER, binding.TILING_PATCH]
@@ -303,3 +304,25 @@ def test_bench_launch_configuration_sampled(cfg, steps):
         assert_close(g, ref, f"config {cfg} step {k}")
         assert torch.equal(out[:B].view(torch.int16), out[B:].view(torch.int16))
     plan.close()
+
+
+def test_step_kernel_selection():
+    """AUTO runs the small-step kernel on steps with one query tile, at most two raster key tiles and little
+    work, the tcgen05 kernel elsewhere; forcing a kernel or patch tiles overrides it."""
+    lib_ready()
+    S, T, M = binding.KERNEL_SIMT, binding.KERNEL_TCGEN05, binding.KERNEL_SMALL
+    plan = binding.Plan(wl.SCALES_256, n_heads=2)
+    assert [plan.step_kernel(k) for k in range(1, 11)] == [M] * 7 + [T] * 3
+    plan.set_kernel(T)
+    assert [plan.step_kernel(k) for k in range(1, 11)] == [T] * 10
+    plan.set_kernel(S)
+    assert [plan.step_kernel(k) for k in range(1, 11)] == [S] * 10
+    plan.close()
+    plan = binding.Plan(wl.SCALES_512, n_heads=2)
+    assert [plan.step_kernel(k) for k in range(1, 11)] == [M] * 6 + [T] * 4
+    plan.close()
+    plan = binding.Plan(wl.SCALES_256, n_heads=2, tiling=binding.TILING_PATCH)
+    assert [plan.step_kernel(k) for k in range(1, 11)] == [T] * 10   # patch query tiles at every step
+    plan.close()
+    with pytest.raises(binding.LitevarError):
+        binding.Plan((1, 2), n_heads=1).step_kernel(3)
