@@ -105,39 +105,54 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
     }
   }
 
-  // ---- stage Q and the K/V prefix (written by earlier work of the stream: wait for it first)
+  // ---- everything that does not read Q, K or V happens before the wait, where it overlaps the tail of the
+  // previous kernel of the stream: kernel parameters into registers (each first touch of a parameter line is
+  // a constant-cache miss), base pointers, zero fill of the padding rows
+  const int n_k = p.n_k, L_k = p.L_k;
+  const uint16_t* qsrc = p.q + b * p.q_sb + h * p.q_sh + (tid & 7) * 8;
+  const uint16_t* ksrc = p.k + b * p.k_sb + h * p.k_sh + (tid & 7) * 8;
+  const uint16_t* vsrc = p.v + b * p.v_sb + h * p.v_sh + (tid & 7) * 8;
+  uint16_t* obase = p.out + b * p.o_sb + h * p.o_sh;
+  int64_t q_st = p.q_st, k_st = p.k_st, v_st = p.v_st, o_st = p.o_st;
+  int64_t o_share = (int64_t)p.share_offset * p.o_sb;
+  float scale_log2 = p.sm_scale * 1.4426950408889634f;
+  asm volatile("" : "+l"(qsrc), "+l"(ksrc), "+l"(vsrc), "+l"(obase));
+  asm volatile("" : "+l"(q_st), "+l"(k_st), "+l"(v_st), "+l"(o_st), "+l"(o_share), "+f"(scale_log2));
+  {
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    for (int c = n_k * 8 + tid; c < q_rows * 8; c += blockDim.x)
+      *reinterpret_cast<uint4*>(Qs + (c >> 3) * kRowPad + (c & 7) * 8) = zero;
+    for (int c = L_k * 8 + tid; c < l_pad * 8; c += blockDim.x) {
+      *reinterpret_cast<uint4*>(Ks + (c >> 3) * kRowPad + (c & 7) * 8) = zero;
+      *reinterpret_cast<uint4*>(Vs + (c >> 3) * kRowPad + (c & 7) * 8) = zero;
+    }
+  }
+
+  // ---- stage Q and the K/V prefix (written by earlier work of the stream: wait for it first).  blockDim is a
+  // multiple of 32, so a thread keeps its 16-byte column (tid % 8) and walks rows.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   {
-    const uint16_t* qbase = p.q + b * p.q_sb + h * p.q_sh;
-    const uint16_t* kbase = p.k + b * p.k_sb + h * p.k_sh;
-    const uint16_t* vbase = p.v + b * p.v_sb + h * p.v_sh;
-    const int total = (q_rows + 2 * l_pad) * 8;
-    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    for (int c = tid; c < total; c += blockDim.x) {
-      int row = c >> 3;
-      const int part = (c & 7) * 8;
-      if (row < q_rows) {
-        uint16_t* dst = Qs + row * kRowPad + part;
-        if (row < p.n_k) cp_async16(dst, qbase + (int64_t)row * p.q_st + part);
-        else *reinterpret_cast<uint4*>(dst) = zero;
-      } else if ((row -= q_rows) < l_pad) {
-        uint16_t* dst = Ks + row * kRowPad + part;
-        if (row < p.L_k) cp_async16(dst, kbase + (int64_t)row * p.k_st + part);
-        else *reinterpret_cast<uint4*>(dst) = zero;
-      } else {
-        row -= l_pad;
-        uint16_t* dst = Vs + row * kRowPad + part;
-        if (row < p.L_k) cp_async16(dst, vbase + (int64_t)row * p.v_st + part);
-        else *reinterpret_cast<uint4*>(dst) = zero;
-      }
-    }
+    const int row_step = (int)(blockDim.x >> 3);
+    uint16_t* kdst = Ks + (tid & 7) * 8;
+    uint16_t* vdst = Vs + (tid & 7) * 8;
+    for (int row = tid >> 3; row < L_k; row += row_step) cp_async16(kdst + row * kRowPad, ksrc + row * k_st);
+    uint16_t* qdst = Qs + (tid & 7) * 8;
+    for (int row = tid >> 3; row < n_k; row += row_step) cp_async16(qdst + row * kRowPad, qsrc + row * q_st);
     asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    // V in a group of its own: the scores of the first round are computed while it is still on its way
+    for (int row = tid >> 3; row < L_k; row += row_step) cp_async16(vdst + row * kRowPad, vsrc + row * v_st);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 1;" ::: "memory");
   }
   __syncthreads();
 
   const int row0 = warp * 16;
-  if (row0 >= p.n_k) return;  // a warp without query rows only helped staging
+  if (row0 >= n_k) {  // a warp without query rows only helped staging
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    return;
+  }
+  bool v_staged = false;
 
   uint32_t qa[4][4];  // Q fragments of the warp's 16 rows, one per 16 head dimensions
 #pragma unroll
@@ -149,7 +164,6 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
   for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
   float lsum[4] = {0.f, 0.f, 0.f, 0.f};  // row sums of P, accumulated by the tensor pipe: P times a block of ones
   float m_run[2] = {-INFINITY, -INFINITY};
-  const float scale_log2 = p.sm_scale * 1.4426950408889634f;
   const uint32_t* m_lo = Ms + (row0 + (lane >> 2)) * 8;  // accumulator rows of this lane: lane / 4 and + 8
   const uint32_t* m_hi = m_lo + 64;
   const int n64 = (l_pad + 63) >> 6;
@@ -181,18 +195,20 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
         }
       }
     }
-    // scores of dead keys are removed
+    // scores of dead keys are removed (groups without a live key are left out altogether)
     const uint32_t bl[2] = {wl[0] >> shift, wl[1] >> shift}, bh[2] = {wh[0] >> shift, wh[1] >> shift};
     float bm[2] = {-INFINITY, -INFINITY};
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
+      if (live[j >> 1]) {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const uint32_t bit = 1u << ((j & 3) * 8 + e);
-        s[j][e] = (bl[j >> 2] & bit) ? s[j][e] : -INFINITY;
-        s[j][2 + e] = (bh[j >> 2] & bit) ? s[j][2 + e] : -INFINITY;
-        bm[0] = fmaxf(bm[0], s[j][e]);
-        bm[1] = fmaxf(bm[1], s[j][2 + e]);
+        for (int e = 0; e < 2; ++e) {
+          const uint32_t bit = 1u << ((j & 3) * 8 + e);
+          s[j][e] = (bl[j >> 2] & bit) ? s[j][e] : -INFINITY;
+          s[j][2 + e] = (bh[j >> 2] & bit) ? s[j][2 + e] : -INFINITY;
+          bm[0] = fmaxf(bm[0], s[j][e]);
+          bm[1] = fmaxf(bm[1], s[j][2 + e]);
+        }
       }
     }
     float alpha[2], m_use[2];
@@ -208,8 +224,15 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
     uint32_t pa[4][4];  // P as A fragments, one per 16 keys
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      pa[j >> 1][(j & 1) * 2] = pack_bf16(ex2(fmaf(s[j][0], scale_log2, -m_use[0])), ex2(fmaf(s[j][1], scale_log2, -m_use[0])));
-      pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(ex2(fmaf(s[j][2], scale_log2, -m_use[1])), ex2(fmaf(s[j][3], scale_log2, -m_use[1])));
+      if (live[j >> 1]) {
+        pa[j >> 1][(j & 1) * 2] = pack_bf16(ex2(fmaf(s[j][0], scale_log2, -m_use[0])), ex2(fmaf(s[j][1], scale_log2, -m_use[0])));
+        pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(ex2(fmaf(s[j][2], scale_log2, -m_use[1])), ex2(fmaf(s[j][3], scale_log2, -m_use[1])));
+      }
+    }
+    if (!v_staged) {  // second block barrier: once per warp, here or after the loop
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncthreads();
+      v_staged = true;
     }
     lsum[0] *= alpha[0];
     lsum[1] *= alpha[0];
@@ -238,6 +261,11 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
     }
   }
 
+  if (!v_staged) {  // no live key in any of the warp's rows (the planner rejects such plans): still join the barrier
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+  }
+
   // ---- normalise, gather the warp's 16 rows in its (now free) Q rows, store 16 bytes per lane
   const float inv[2] = {1.f / lsum[0], 1.f / lsum[2]};
   __syncwarp();
@@ -251,16 +279,15 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
     }
   }
   __syncwarp();
-  uint16_t* obase = p.out + b * p.o_sb + h * p.o_sh;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int c = i * 32 + lane;
     const int row = row0 + (c >> 3), part = (c & 7) * 8;
-    if (row < p.n_k) {
+    if (row < n_k) {
       const uint4 v = *reinterpret_cast<const uint4*>(Qs + row * kRowPad + part);
-      uint16_t* dst = obase + (int64_t)row * p.o_st + part;
+      uint16_t* dst = obase + row * o_st + part;
       *reinterpret_cast<uint4*>(dst) = v;
-      if (p.share_offset > 0) *reinterpret_cast<uint4*>(dst + (int64_t)p.share_offset * p.o_sb) = v;
+      if (o_share != 0) *reinterpret_cast<uint4*>(dst + o_share) = v;
     }
   }
 }
