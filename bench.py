@@ -433,6 +433,14 @@ def gpu_arm(args):
     if barrier:
         barrier()
     pk = peaks()
+    if args.calibration:
+        # the window calibration kernel alone (for profiler runs); one GPU
+        if rank == 0:
+            print(json.dumps({"calibration": measure_calibration(device, pk), "peaks": pk}), flush=True)
+        if barrier:
+            barrier()
+            torch.distributed.destroy_process_group()
+        return
     w = wl.WORKLOADS[args.config]
     variant = "dense" if args.dense else "window"
 
@@ -526,6 +534,7 @@ def gpu_arm(args):
                        "avg_launch_us": round(avg_launch_s * 1e6, 3),
                        "other_kernels": [
                            {"kernel": n, "steps": t["steps"], "launches_per_generation": t["launches"],
+                            "algorithmic_bytes_per_launch": round(t["bytes"] / t["launches"]),
                             "avg_launch_us": round(t["us"] / t["launches"], 3),
                             "share_of_generation_time": round(t["us"] / total_us, 4),
                             "hbm_frac": round(t["bytes"] / (t["us"] * 1e-6) / 1e9 / pk["hbm"], 4)}
@@ -675,6 +684,7 @@ def main():
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed graph replays (for profiler runs): no eager, end-to-end, "
                          "CPU or all-workload legs")
+    ap.add_argument("--calibration", action="store_true", help="only the window calibration kernel's figures")
     ap.add_argument("--rho", type=int, nargs=2, default=None, help="window radius ratio num den (default: the workload's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
