@@ -24,12 +24,23 @@ What follows the paper, and where:
 * R_0 = 1   -- Section 2: the mask degenerates to full attention.
 * ASC       -- Section 3: the unconditional CFG branch reuses the conditional branch's
   attention output.
+* QKV8      -- Section 4: Q, K and V are quantised to 8-bit integers with a scale s and a
+  zero point z taken online from the maximum and minimum of the data (dynamic
+  quantisation), x_q = round(clamp((x - z) / s, -2^(B-1), 2^(B-1))), z = (max + min) / 2.
+  Readings: one (s, z) per token row of a head (64 values); s = (max - min) / (2^B - 1),
+  the step that makes the stated clamp range the range of the data (the printed
+  s = max(abs(x)) does not match the printed clamp bounds); the upper clamp bound is
+  2^(B-1) - 1 so that the code fits B bits; round = to nearest, ties to even; the
+  attention then runs on the dequantised values x_q * s + z, rounded to bf16.
 
 Parity status: mask, schedule, softmax-attention and ASC are pinned by the CPU tests
 (paper's worked shapes, Table 1's saving, library softmax attention, brute force in
 exact rationals, closed-form counts).  The numeric window widths that the paper
 obtains by calibrating on VAR activations are NOT reproducible here (needs weights
 and ImageNet): for those, parity unpinned; the default rule below is a stand-in.
+The row quantiser is pinned by a hand-worked row, the classical unsigned min-max
+formula, its error bound and its invariances; which granularity and step the authors
+used is a reading (see above), not something the paper fixes.
 """
 from __future__ import annotations
 
@@ -245,6 +256,35 @@ def calibrate_radius(scales: Sequence[int], k: int, maps: np.ndarray, r0: float,
             w += 1
         out[j - 1] = w
     return out
+
+
+# ----------------------------------------------------------------------------- 8-bit Q/K/V
+def round_to_bf16(x32: np.ndarray) -> np.ndarray:
+    """fp32 -> nearest bf16 (ties to even), returned as fp32 holding the bf16 value."""
+    u = np.asarray(x32, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) >> 16 << 16
+    return u.astype(np.uint32).view(np.float32)
+
+
+def quantize_rows(x: np.ndarray, bits: int = 8):
+    """Dynamic min-max quantisation of Section 4, one (s, z) per row (last axis).
+
+    The decision which integer a value becomes is taken in fp32, one IEEE operation at a time, in the
+    order written here: z = (max + min) * 0.5; s = (max - min) / (2^B - 1);
+    code = clamp(rint((x - z) / s), -2^(B-1), 2^(B-1) - 1); dequantised = bf16(code * s + z).
+    A constant row (s = 0) has code 0 everywhere and dequantises to z.
+    Returns (codes int32, s fp32 [..., 1], z fp32 [..., 1], dequantised fp32 holding bf16 values)."""
+    x = np.asarray(x, dtype=np.float32)
+    mx = x.max(axis=-1, keepdims=True)
+    mn = x.min(axis=-1, keepdims=True)
+    z = (mx + mn) * np.float32(0.5)
+    s = (mx - mn) / np.float32(2 ** bits - 1)
+    safe = np.where(s > 0, s, np.float32(1))
+    code = np.rint((x - z) / safe)
+    code = np.clip(code, -(2 ** (bits - 1)), 2 ** (bits - 1) - 1)
+    code = np.where(s > 0, code, np.float32(0)).astype(np.float32)
+    deq = round_to_bf16((code * s).astype(np.float32) + z)
+    return code.astype(np.int32), s, z, deq
 
 
 # ----------------------------------------------------------------------------- attention

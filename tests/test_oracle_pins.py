@@ -498,3 +498,67 @@ def test_sampled_rows_match_full_evaluation():
     got = orc.attention_sampled(scales, k, w[k - 1], Q, Kc, Vc, samples, share_cfg=True)
     for i, (b, h, q) in enumerate(samples):
         assert np.abs(got[i] - full[b, h, q]).max() < 1e-13
+
+
+# ----------------------------------------------------------------------------- 8-bit Q/K/V (Section 4)
+def test_quantizer_hand_worked_row_with_ties():
+    # max = 255, min = 0: z = 127.5 and s = 1 exactly, so (x - z) / s = x - 127.5 is a tie for every integer x
+    # and rounds to the even neighbour: x - 128 when that is even, else x - 127; the top value clamps to 127.
+    x = np.arange(256, dtype=np.float32)[None]
+    code, s, z, deq = orc.quantize_rows(x)
+    assert s.item() == 1.0 and z.item() == 127.5
+    want = [xi - 128 if (xi - 128) % 2 == 0 else xi - 127 for xi in range(256)]
+    want[255] = 127
+    assert code[0].tolist() == want
+    assert code.min() == -128 and code.max() == 127
+    # dequantised = code + 127.5, which lies half-way between two bf16 values from 128 on (bf16 spacing 1)
+    assert deq[0, :4].tolist() == [-0.5, 1.5, 1.5, 3.5]
+    assert deq[0, 255] == 254.0 and deq[0, 254] == 254.0
+
+
+def test_quantizer_is_the_textbook_mid_rise_quantiser_between_ties():
+    # away from ties the code is floor((x - min) / s) - 127: 255 cells of width s, reconstructed at their centres
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((500, 64)).astype(np.float32)
+    code, s, z, deq = orc.quantize_rows(x)
+    x64, mn, mx = x.astype(np.float64), x.min(-1, keepdims=True).astype(np.float64), x.max(-1, keepdims=True).astype(np.float64)
+    y = (x64 - mn) / ((mx - mn) / 255.0)
+    clear = np.abs(y - np.rint(y)) > 1e-3          # not within fp32 noise of a cell boundary
+    assert clear.mean() > 0.95
+    assert np.array_equal(code[clear], (np.floor(y) - 127).astype(np.int32)[clear])
+    # error bound of a uniform quantiser: half a step (plus the fp32 noise of s and z), before the bf16 rounding
+    rec = code.astype(np.float64) * s.astype(np.float64) + z.astype(np.float64)
+    assert np.all(np.abs(rec - x64) <= 0.5 * s.astype(np.float64) * (1 + 1e-5) + 1e-6)
+    # after it: at most half a bf16 spacing more
+    assert np.all(np.abs(deq.astype(np.float64) - rec) <= np.abs(rec) * 2.0 ** -8 + 1e-30)
+    # the extremes sit on the ties +-127.5: the maximum always ends at 127 (128 is clamped), the minimum at
+    # -128 or, when fp32 rounding of s and z leaves it a hair inside, at -127
+    assert np.all(code[np.arange(500), x.argmax(-1)] == 127)
+    assert np.all(np.isin(code[np.arange(500), x.argmin(-1)], (-128, -127)))
+
+
+def test_quantizer_invariances_and_degenerate_rows():
+    rng = np.random.default_rng(6)
+    x = rng.standard_normal((64, 64)).astype(np.float32)
+    code, s, z, _ = orc.quantize_rows(x)
+    c4, s4, z4, _ = orc.quantize_rows(x * np.float32(4))          # power-of-two scaling is exact in fp32
+    assert np.array_equal(c4, code) and np.array_equal(s4, s * 4) and np.array_equal(z4, z * 4)
+    cn, _, zn, _ = orc.quantize_rows(-x)                            # mirror image away from ties and clamps
+    y = (x.astype(np.float64) - x.min(-1, keepdims=True)) / ((x.max(-1, keepdims=True) - x.min(-1, keepdims=True)) / 255.0)
+    clear = np.abs(y - np.rint(y)) > 1e-3
+    assert np.array_equal(cn[clear], -code[clear]) and np.array_equal(zn, -z)
+    const = np.full((3, 64), 1.375, np.float32)
+    cc, sc, zc, dc = orc.quantize_rows(const)
+    assert not cc.any() and not sc.any() and np.array_equal(dc, const)
+    for bits in (4, 6):                                              # fewer levels, same rule
+        cb, sb, _, _ = orc.quantize_rows(x, bits)
+        assert cb.min() in (-2 ** (bits - 1), -2 ** (bits - 1) + 1) and cb.max() == 2 ** (bits - 1) - 1
+        assert np.allclose(sb, (x.max(-1, keepdims=True) - x.min(-1, keepdims=True)) / (2 ** bits - 1), rtol=1e-6)
+
+
+def test_round_to_bf16_matches_library_rounding():
+    rng = np.random.default_rng(7)
+    x = np.concatenate([rng.standard_normal(4096).astype(np.float32) * np.float32(37.0),
+                        np.array([1.00390625, 1.01171875, 254.5, 255.5, -3.0e-40, 0.0], np.float32)])
+    want = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(orc.round_to_bf16(x), want)
