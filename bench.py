@@ -411,6 +411,65 @@ def measure_calibration(device, pk):
     return rows
 
 
+def measure_qkv8(device, pk):
+    """8-bit Q/K/V (paper Section 4).  (1) The row quantiser alone on a K cache of workload 3's shape against
+    the HBM roofline (every row read once and written once).  (2) Workload 2's generation with the step's Q
+    and appended K/V rows quantised in place before every attention call (one extra launch per call)."""
+    from paper_2411_17178_b200 import binding
+    w3 = wl.WORKLOADS[3]
+    shape = (2 * w3.batch_pairs, w3.n_heads, wl.cache_len(w3.scales, 10), wl.HEAD_DIM)
+    x = device_randn_bf16(shape, 77, device)
+    y = torch.empty_like(x)
+    for _ in range(3):
+        binding.quantize_rows(x, 8, out=y)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(10):
+        binding.quantize_rows(x, 8, out=y)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 10
+    nbytes = 2 * x.numel() * 2
+    res = {"quantiser": {"tensor": list(shape), "bytes_read_plus_written": nbytes, "us_per_call": round(ms * 1e3, 2),
+                         "gbs": round(nbytes / ms / 1e6, 1), "hbm_frac": round(nbytes / ms / 1e6 / pk["hbm"], 4)}}
+    del x, y
+    w = wl.WORKLOADS[2]
+    plan = make_plan(w, "window")
+    n_sets, _ = sets_needed(w)
+    bufs = Buffers(w, n_sets, device)
+    off = [0]
+    for s_ in w.scales:
+        off.append(off[-1] + s_ * s_)
+    calls = generation_calls(w, n_sets, max(w.n_layers, n_sets))
+
+    def generation():
+        for k, s_ in calls:
+            binding.quantize_qkv(bufs.q[s_][k], bufs.k[s_][:, :, off[k - 1]:off[k]], bufs.v[s_][:, :, off[k - 1]:off[k]])
+            plan.forward(k, w.batch_pairs, bufs.q[s_][k], bufs.k[s_], bufs.v[s_], bufs.out[s_][k])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        generation()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        generation()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(20):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    res["workload2_generation_us_with_quantised_qkv"] = round(e0.elapsed_time(e1) / 20 * 1e3 * w.n_layers / max(w.n_layers, n_sets), 2)
+    res["launches_per_generation"] = 2 * len(w.steps) * w.n_layers
+    assert plan.poll() == 0
+    plan.close()
+    return res
+
+
 def gpu_arm(args):
     from paper_2411_17178_b200 import build as lvbuild
     rank = int(os.environ.get("RANK", "0"))
@@ -436,7 +495,8 @@ def gpu_arm(args):
     if args.calibration:
         # the window calibration kernel alone (for profiler runs); one GPU
         if rank == 0:
-            print(json.dumps({"calibration": measure_calibration(device, pk), "peaks": pk}), flush=True)
+            print(json.dumps({"calibration": measure_calibration(device, pk), "qkv8": measure_qkv8(device, pk),
+                              "peaks": pk}), flush=True)
         if barrier:
             barrier()
             torch.distributed.destroy_process_group()
@@ -574,6 +634,7 @@ def gpu_arm(args):
             torch.cuda.empty_cache()
         out["all_configs"] = table
         out["calibration"] = measure_calibration(device, pk)
+        out["qkv8"] = measure_qkv8(device, pk)
     print(json.dumps(out), flush=True)
 
 
@@ -684,7 +745,7 @@ def main():
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed graph replays (for profiler runs): no eager, end-to-end, "
                          "CPU or all-workload legs")
-    ap.add_argument("--calibration", action="store_true", help="only the window calibration kernel's figures")
+    ap.add_argument("--calibration", action="store_true", help="only the figures of the window calibration and row quantiser kernels")
     ap.add_argument("--rho", type=int, nargs=2, default=None, help="window radius ratio num den (default: the workload's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

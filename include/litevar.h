@@ -244,6 +244,40 @@ litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel);
  * LITEVAR_KERNEL_SIMT, _TCGEN05 or _SMALL.  Host only; the paper has no counterpart (it gives no kernel design). */
 litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t* kernel);
 
+/*
+ * 8-bit Q/K/V (paper Section 4, dynamic quantisation): quantise every token row of a head (head_dim values) of
+ * a bf16 tensor x[batch][n_heads][n_tokens][head_dim] (element strides sx, head_dim contiguous) to `bits`-bit
+ * integers with a scale and a zero point taken from the row's maximum and minimum:
+ *     z = (max + min) / 2,  s = (max - min) / (2^bits - 1),
+ *     code = clamp(round((x - z) * r), -2^(bits-1), 2^(bits-1) - 1), r = 1 / s   (round to nearest even; s = 0:
+ *     code 0), all in fp32, one IEEE operation at a time.  Outputs, each optional (NULL = not wanted), all device memory:
+ *   x_dq   bf16, strides sdq: the dequantised rows code * s + z rounded to bf16 - what the attention then reads;
+ *          may be x itself (in place)
+ *   codes  int8 [batch][n_heads][n_tokens][head_dim], dense, 8-byte aligned
+ *   scale, zero  fp32 [batch][n_heads][n_tokens], dense
+ * Granularity (per token row) and the step s are readings of the paper, which prints s = max(abs(x)) beside
+ * clamp bounds that do not match it.  Asynchronous on `stream`, allocates nothing, graph-capturable.
+ * Errors: NULL x, bad strides or alignment, batch / n_heads / n_tokens < 1, bits outside 2..8 -> INVALID_ARG;
+ * head_dim != 64 -> UNSUPPORTED.  Pointers are borrowed.
+ */
+litevar_status_t litevar_quantize_rows(const void* x, const litevar_strides_t* sx, int32_t batch, int32_t n_heads,
+                                       int32_t n_tokens, int32_t head_dim, int32_t bits, void* x_dq,
+                                       const litevar_strides_t* sdq, int8_t* codes, float* scale, float* zero,
+                                       void* stream);
+
+/*
+ * The same quantiser for the three tensors of one attention call, in place, in one launch: the step's Q
+ * (n_q_tokens rows per head) and the K and V rows appended to the cache at this step (n_kv_tokens rows per head
+ * each; pass pointers to the first appended row).  Every row is replaced by its dequantised value, which is what
+ * litevar_attn_forward then reads (paper Section 4: Q, K and V in attention quantised to 8 bits).  Launched
+ * with programmatic stream serialisation, so that its launch overlaps the previous kernel of the stream; it
+ * waits for that kernel before it reads.  Errors as litevar_quantize_rows.
+ */
+litevar_status_t litevar_quantize_qkv(void* q, const litevar_strides_t* sq, int32_t n_q_tokens, void* k,
+                                      const litevar_strides_t* sk, void* v, const litevar_strides_t* sv,
+                                      int32_t n_kv_tokens, int32_t batch, int32_t n_heads, int32_t head_dim,
+                                      int32_t bits, void* stream);
+
 /* Frees the plan and its device buffers.  NULL is allowed. */
 void litevar_plan_destroy(litevar_plan_t* plan);
 

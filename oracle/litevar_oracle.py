@@ -270,8 +270,9 @@ def quantize_rows(x: np.ndarray, bits: int = 8):
     """Dynamic min-max quantisation of Section 4, one (s, z) per row (last axis).
 
     The decision which integer a value becomes is taken in fp32, one IEEE operation at a time, in the
-    order written here: z = (max + min) * 0.5; s = (max - min) / (2^B - 1);
-    code = clamp(rint((x - z) / s), -2^(B-1), 2^(B-1) - 1); dequantised = bf16(code * s + z).
+    order written here: z = (max + min) * 0.5; s = (max - min) / (2^B - 1); r = 1 / s;
+    code = clamp(rint((x - z) * r), -2^(B-1), 2^(B-1) - 1); dequantised = bf16(code * s + z).
+    (The division by s is taken as a multiplication by the row's reciprocal step, one division per row.)
     A constant row (s = 0) has code 0 everywhere and dequantises to z.
     Returns (codes int32, s fp32 [..., 1], z fp32 [..., 1], dequantised fp32 holding bf16 values)."""
     x = np.asarray(x, dtype=np.float32)
@@ -280,7 +281,8 @@ def quantize_rows(x: np.ndarray, bits: int = 8):
     z = (mx + mn) * np.float32(0.5)
     s = (mx - mn) / np.float32(2 ** bits - 1)
     safe = np.where(s > 0, s, np.float32(1))
-    code = np.rint((x - z) / safe)
+    r = np.float32(1) / safe
+    code = np.rint((x - z) * r)
     code = np.clip(code, -(2 ** (bits - 1)), 2 ** (bits - 1) - 1)
     code = np.where(s > 0, code, np.float32(0)).astype(np.float32)
     deq = round_to_bf16((code * s).astype(np.float32) + z)

@@ -25,6 +25,7 @@ TILING_AUTO, TILING_RASTER, TILING_PATCH = 0, 1, 2
 
 EXPORTS = (
     "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_static", "litevar_calibrate_windows",
+    "litevar_quantize_rows", "litevar_quantize_qkv",
     "litevar_plan_stats", "litevar_plan_tile_counts",
     "litevar_plan_export_tiles", "litevar_plan_export_bounds", "litevar_plan_materialize_mask",
     "litevar_plan_poll_device_status", "litevar_plan_set_kernel", "litevar_plan_step_kernel", "litevar_plan_destroy",
@@ -80,6 +81,12 @@ def load() -> ctypes.CDLL:
                                                 P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides), P]
     lib.litevar_calibrate_windows.restype = ctypes.c_int
     lib.litevar_calibrate_windows.argtypes = [ctypes.POINTER(I32), I32, I32, I32, P, I64, ctypes.c_float, P, P, P]
+    lib.litevar_quantize_rows.restype = ctypes.c_int
+    lib.litevar_quantize_rows.argtypes = [P, ctypes.POINTER(_Strides), I32, I32, I32, I32, I32, P,
+                                          ctypes.POINTER(_Strides), P, P, P, P]
+    lib.litevar_quantize_qkv.restype = ctypes.c_int
+    lib.litevar_quantize_qkv.argtypes = [P, ctypes.POINTER(_Strides), I32, P, ctypes.POINTER(_Strides), P,
+                                         ctypes.POINTER(_Strides), I32, I32, I32, I32, I32, P]
     lib.litevar_plan_stats.restype = ctypes.c_int
     lib.litevar_plan_stats.argtypes = [P, I32, I32] + [ctypes.POINTER(I64)] * 4
     lib.litevar_plan_tile_counts.restype = ctypes.c_int
@@ -303,6 +310,42 @@ def calibrate_windows(scales: Sequence[int], step_k: int, maps, r0: float, n_glo
                                        ratio.ctypes.data if want_ratio else None, _stream_ptr(stream))
     _check(st, "litevar_calibrate_windows")
     return (rad, ratio) if want_ratio else rad
+
+
+def quantize_rows(x, bits: int = 8, out=None, want_codes: bool = False, stream=None):
+    """litevar_quantize_rows on a CUDA bf16 tensor [batch, heads, tokens, 64] (last dimension contiguous).
+    Writes the dequantised rows to `out` (bf16, same shape; `x` itself for in place; a new tensor when None)
+    and returns it, or (out, codes int8, scale fp32, zero fp32) when `want_codes`."""
+    import torch
+    lib = load()
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 4 and x.stride(3) == 1
+    if out is None:
+        out = torch.empty(x.shape, dtype=torch.bfloat16, device=x.device)
+    assert out.is_cuda and out.dtype == torch.bfloat16 and out.shape == x.shape and out.stride(3) == 1
+    B, H, T, D = x.shape
+    codes = scale = zero = None
+    if want_codes:
+        codes = torch.empty((B, H, T, D), dtype=torch.int8, device=x.device)
+        scale = torch.empty((B, H, T), dtype=torch.float32, device=x.device)
+        zero = torch.empty((B, H, T), dtype=torch.float32, device=x.device)
+    st = lib.litevar_quantize_rows(x.data_ptr(), ctypes.byref(_strides(x)), B, H, T, D, int(bits), out.data_ptr(),
+                                   ctypes.byref(_strides(out)), codes.data_ptr() if want_codes else None,
+                                   scale.data_ptr() if want_codes else None,
+                                   zero.data_ptr() if want_codes else None, _stream_ptr(stream))
+    _check(st, "litevar_quantize_rows")
+    return (out, codes, scale, zero) if want_codes else out
+
+
+def quantize_qkv(q, k_new, v_new, bits: int = 8, stream=None) -> None:
+    """litevar_quantize_qkv: quantise-dequantise, in place and in one launch, the step's Q [batch, heads, n_k, 64]
+    and the appended cache rows k_new, v_new [batch, heads, n_new, 64] (views into the caches)."""
+    lib = load()
+    B, H, Tq, D = q.shape
+    assert k_new.shape == v_new.shape and k_new.shape[:2] == (B, H) and k_new.shape[3] == D
+    st = lib.litevar_quantize_qkv(q.data_ptr(), ctypes.byref(_strides(q)), Tq, k_new.data_ptr(),
+                                  ctypes.byref(_strides(k_new)), v_new.data_ptr(), ctypes.byref(_strides(v_new)),
+                                  int(k_new.shape[2]), B, H, D, int(bits), _stream_ptr(stream))
+    _check(st, "litevar_quantize_qkv")
 
 
 def status_string(status: int) -> str:
