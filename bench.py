@@ -264,62 +264,66 @@ def time_eager(plan, w, bufs, calls, steps, warmup):
 
 
 def time_e2e(plan, w: wl.Workload, steps, warmup, device):
-    """Per-call API with host buffers: H2D of the call's Q and of the new scale's K/V rows (only the
-    batch rows the call computes), forward, D2H of the call's output.  One layer's device cache is
-    reused for every layer (the copies and the calls are the same)."""
+    """Per-call API with host buffers.  Every call uploads one pinned block [Q | new K rows | new V rows] (only
+    the batch rows the call computes) on an upload stream, appends the K/V rows to the device cache with one
+    device copy, runs the forward (Q is read from the uploaded block) and sends the output back on a third
+    stream, so that the uploads, the kernels and the downloads of neighbouring calls overlap (the link is
+    full duplex).  Staging and output buffers alternate between two sets.  One layer's device cache is reused
+    for every layer (the copies and the calls are the same)."""
     rows = 2 * w.batch_pairs
     share = w.share_cfg
     comp = w.batch_pairs if share else rows
     L = wl.cache_len(w.scales, max(w.steps))
     H, D = w.n_heads, wl.HEAD_DIM
     host_k, host_v = wl.make_kv(w, 0)
-    host_q = {k: wl.make_q(w, 0, k).pin_memory() for k in w.steps}
-    host_out = {k: torch.empty_like(host_q[k]).pin_memory() for k in w.steps}
-    dk = torch.zeros((rows, H, L, D), dtype=torch.bfloat16, device=device)
-    dv = torch.zeros_like(dk)
-    dq = {k: torch.empty((rows, H, w.scales[k - 1] ** 2, D), dtype=torch.bfloat16, device=device) for k in w.steps}
-    do = {k: torch.empty_like(dq[k]) for k in w.steps}
     off = [0]
     for s in w.scales:
         off.append(off[-1] + s * s)
+    n_tok = {k: w.scales[k - 1] ** 2 for k in w.steps}
+    host_in = {k: torch.stack([wl.make_q(w, 0, k)[:comp], host_k[:comp, :, off[k - 1]:off[k]],
+                               host_v[:comp, :, off[k - 1]:off[k]]]).contiguous().pin_memory() for k in w.steps}
+    host_out = {k: torch.empty((rows, H, n_tok[k], D), dtype=torch.bfloat16).pin_memory() for k in w.steps}
+    dkv = torch.zeros((2, rows, H, L, D), dtype=torch.bfloat16, device=device)
+    dk, dv = dkv[0], dkv[1]
     if min(w.steps) > 1:  # single-step workloads: the earlier scales are already cached on the device
         a = off[min(w.steps) - 1]
         dk[:, :, :a].copy_(host_k[:, :, :a])
         dv[:, :, :a].copy_(host_v[:, :, :a])
-    # the rows a call appends to the cache, contiguous in pinned host memory
-    new_k = {k: host_k[:comp, :, off[k - 1]:off[k]].contiguous().pin_memory() for k in w.steps}
-    new_v = {k: host_v[:comp, :, off[k - 1]:off[k]].contiguous().pin_memory() for k in w.steps}
+    stage = {k: [torch.empty((3, comp, H, n_tok[k], D), dtype=torch.bfloat16, device=device) for _ in range(2)]
+             for k in w.steps}
+    outs = {k: [torch.empty((rows, H, n_tok[k], D), dtype=torch.bfloat16, device=device) for _ in range(2)]
+            for k in w.steps}
     h2d = d2h = 0
     for k in w.steps:
-        n_k = w.scales[k - 1] ** 2
-        h2d += w.n_layers * comp * H * n_k * D * 2 * 3
-        d2h += w.n_layers * rows * H * n_k * D * 2
-
-    # results travel back on a second stream, so a call's device-to-host copy overlaps the next call's
-    # host-to-device copies (the link is full duplex); two output buffers per step alternate
-    main, back = torch.cuda.current_stream(), torch.cuda.Stream()
-    do2 = {k: (do[k], torch.empty_like(do[k])) for k in w.steps}
-    freed = {k: [None, None] for k in w.steps}
+        h2d += w.n_layers * host_in[k].numel() * 2
+        d2h += w.n_layers * host_out[k].numel() * 2
+    main, back, up = torch.cuda.current_stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev = {k: [[torch.cuda.Event() for _ in range(3)] for _ in range(2)] for k in w.steps}  # uploaded, computed, downloaded
 
     def generation():
+        used = {k: [False, False] for k in w.steps}
         for k in w.steps:
             a, b = off[k - 1], off[k]
             for layer in range(w.n_layers):
                 i = layer & 1
-                if freed[k][i] is not None:
-                    main.wait_event(freed[k][i])
-                dq[k][:comp].copy_(host_q[k][:comp], non_blocking=True)
-                dk[:comp, :, a:b].copy_(new_k[k], non_blocking=True)
-                dv[:comp, :, a:b].copy_(new_v[k], non_blocking=True)
-                plan.forward(k, w.batch_pairs, dq[k], dk, dv, do2[k][i])
-                done = torch.cuda.Event()
-                done.record(main)
-                back.wait_event(done)
+                st, (uploaded, computed, downloaded) = stage[k][i], ev[k][i]
+                if used[k][i]:
+                    up.wait_event(computed)       # the staging block was read by the call two layers ago
+                    main.wait_event(downloaded)   # and its output buffer has gone back to the host
+                with torch.cuda.stream(up):
+                    st.copy_(host_in[k], non_blocking=True)
+                    uploaded.record(up)
+                main.wait_event(uploaded)
+                dkv[:, :comp, :, a:b].copy_(st[1:3])
+                plan.forward(k, w.batch_pairs, st[0], dk, dv, outs[k][i])
+                computed.record(main)
+                back.wait_event(computed)
                 with torch.cuda.stream(back):
-                    host_out[k].copy_(do2[k][i], non_blocking=True)
-                    freed[k][i] = torch.cuda.Event()
-                    freed[k][i].record(back)
+                    host_out[k].copy_(outs[k][i], non_blocking=True)
+                    downloaded.record(back)
+                used[k][i] = True
         main.wait_stream(back)
+        main.wait_stream(up)
 
     for _ in range(warmup):
         generation()
