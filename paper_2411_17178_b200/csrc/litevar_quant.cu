@@ -104,7 +104,12 @@ __global__ void __launch_bounds__(kQuantThreads) quant_rows_kernel(QuantArgs a) 
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       float q = 0.f;
-      if (s > 0.f) q = fminf(fmaxf(rintf(__fmul_rn(__fsub_rn(v[i], z), r)), a.lo), a.hi);
+      if (s > 0.f) {
+        // round to nearest even without the conversion pipe: adding and subtracting 1.5 * 2^23 is exact
+        // rounding to an integer for |y| < 2^22, and |y| stays near 2^(B-1) here
+        const float y = __fmul_rn(__fsub_rn(v[i], z), r);
+        q = fminf(fmaxf(__fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f), a.lo), a.hi);
+      }
       c[i] = q;
     }
 #pragma unroll
