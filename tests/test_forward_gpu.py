@@ -326,3 +326,35 @@ def test_step_kernel_selection():
     plan.close()
     with pytest.raises(binding.LitevarError):
         binding.Plan((1, 2), n_heads=1).step_kernel(3)
+
+
+@pytest.mark.parametrize("scales,n_global,share", [
+    ((1, 11), 0, False),        # 121 queries (eight warps, the last with 9 rows) x 122 keys
+    ((15, 4), 0, True),         # 16 queries x 241 keys: one warp, four 64-key rounds, two key tiles, shared step
+    ((2, 9, 3), 1, False),      # non-monotone scales: 9 queries x 94 keys at the last step
+    ((1, 2, 3, 4, 6, 9, 5), 3, True),   # 25 queries x 172 keys with windows on four scales
+    ((12, 8), 0, False),        # 64 queries x 208 keys: 4 warps x 4 rounds
+])
+def test_small_step_kernel_shape_extremes(scales, n_global, share):
+    """Shapes at the edges of what the small-step kernel takes (row groups and key rounds with ragged ends,
+    the largest eligible warp x round products), each step checked in full against the oracle."""
+    lib_ready()
+    H, B = 3, 1
+    w = wl.small_workload(scales, n_heads=H, batch_pairs=B, share_cfg=share, index=90)
+    plan = binding.Plan(scales, n_heads=H, n_global_scales=n_global,
+                        share_steps=[1] * len(scales) if share else None)
+    tab = orc.window_table(scales, n_global_scales=n_global)
+    Kc, Vc = wl.make_kv(w, 0)
+    for k in range(1, len(scales) + 1):
+        n_k, L_k = orc.map_shape(scales, k)
+        small = n_k <= 128 and L_k <= 256 and -(-n_k // 16) * -(-L_k // 64) <= 18
+        assert plan.step_kernel(k) == (binding.KERNEL_SMALL if small else binding.KERNEL_TCGEN05), (scales, k)
+        assert small or k < len(scales)     # the step each case is about runs on the small-step kernel
+        assert np.array_equal(plan.materialize_mask(k), orc.mask(scales, k, tab[k - 1]))
+        Q = wl.make_q(w, 0, k)
+        got, out = run_forward(plan, k, B, Q, Kc, Vc)
+        ref = orc.attention_step(scales, k, tab[k - 1], Q, Kc, Vc, share_cfg=share)
+        assert_close(got, ref, f"small-step kernel scales={scales} step {k}")
+        if share:
+            assert torch.equal(out[:B].view(torch.int16), out[B:].view(torch.int16))
+    plan.close()
