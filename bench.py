@@ -379,7 +379,7 @@ def measure_config(w: wl.Workload, variant: str, rho, steps, warmup, device, pk,
             ms_k = time_graph(plan, w, bufs, [(k, layer % n_sets) for layer in range(repeat)], max(2, steps // 2), 2)
             per_step[str(k)] = round(ms_k * 1e3 / repeat, 2)
         res["us_per_call_by_step"] = per_step
-        res["kernel_by_step"] = {str(k): KERNEL_NAMES[plan.step_kernel(k)] for k in w.steps}
+        res["kernel_by_step"] = {str(k): KERNEL_NAMES[plan.step_kernel(k, w.batch_pairs)] for k in w.steps}
     plan.close()
     return res, bufs
 
@@ -575,7 +575,7 @@ def gpu_arm(args):
     # with the larger share of the generation is the one reported.
     groups = {}
     for k in w.steps:
-        groups.setdefault(KERNEL_NAMES[plan.step_kernel(k)], []).append(k)
+        groups.setdefault(KERNEL_NAMES[plan.step_kernel(k, w.batch_pairs)], []).append(k)
     timed = {}
     for name, ks in groups.items():
         g_calls = [(k, layer % n_sets) for k in ks for layer in range(repeat)]

@@ -240,9 +240,10 @@ litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan);
  * forwards. */
 litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel);
 
-/* Which kernel litevar_attn_forward launches for step_k under the current selection: *kernel receives
- * LITEVAR_KERNEL_SIMT, _TCGEN05 or _SMALL.  Host only; the paper has no counterpart (it gives no kernel design). */
-litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t* kernel);
+/* Which kernel litevar_attn_forward launches for step_k with batch_pairs under the current selection:
+ * *kernel receives LITEVAR_KERNEL_SIMT, _TCGEN05 or _SMALL.  Host only; the paper has no counterpart (it gives no kernel design). */
+litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
+                                          int32_t* kernel);
 
 /*
  * 8-bit Q/K/V (paper Section 4, dynamic quantisation): quantise every token row of a head (head_dim values) of

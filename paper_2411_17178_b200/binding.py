@@ -102,7 +102,7 @@ def load() -> ctypes.CDLL:
     lib.litevar_plan_set_kernel.restype = ctypes.c_int
     lib.litevar_plan_set_kernel.argtypes = [P, I32]
     lib.litevar_plan_step_kernel.restype = ctypes.c_int
-    lib.litevar_plan_step_kernel.argtypes = [P, I32, ctypes.POINTER(I32)]
+    lib.litevar_plan_step_kernel.argtypes = [P, I32, I32, ctypes.POINTER(I32)]
     lib.litevar_plan_destroy.restype = None
     lib.litevar_plan_destroy.argtypes = [P]
     lib.litevar_status_string.restype = ctypes.c_char_p
@@ -256,10 +256,11 @@ class Plan:
     def set_kernel(self, kernel: int) -> None:
         _check(self._lib.litevar_plan_set_kernel(self._h, int(kernel)), "litevar_plan_set_kernel")
 
-    def step_kernel(self, step_k: int) -> int:
-        """KERNEL_SIMT, KERNEL_TCGEN05 or KERNEL_SMALL: what a forward of this step launches."""
+    def step_kernel(self, step_k: int, batch_pairs: int = 1) -> int:
+        """KERNEL_SIMT, KERNEL_TCGEN05 or KERNEL_SMALL: what a forward of this step with that batch launches."""
         out = ctypes.c_int32(0)
-        _check(self._lib.litevar_plan_step_kernel(self._h, int(step_k), ctypes.byref(out)), "litevar_plan_step_kernel")
+        _check(self._lib.litevar_plan_step_kernel(self._h, int(step_k), int(batch_pairs), ctypes.byref(out)),
+               "litevar_plan_step_kernel")
         return int(out.value)
 
 

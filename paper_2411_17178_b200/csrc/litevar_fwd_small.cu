@@ -25,6 +25,8 @@ namespace {
 
 constexpr int kRowPad = 72;        // bf16 elements per staged row: 144 B keeps ldmatrix rows on distinct banks
 constexpr int kSmallMaxWarps = 8;  // 16 query rows each
+constexpr int kMergePad = 68;      // floats per row of a partial output handed from one warp of a pair to the other
+constexpr int kMergeFloats = 16 * kMergePad + 32;  // per row group: 16 partial output rows, 16 maxima, 16 sums
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -64,7 +66,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
-__global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParams p, SmallLists lists) {
+// SPLIT = 1: one warp per 16 query rows.  SPLIT = 2: two warps per 16 query rows, each taking every other
+// 64-key round, merged through shared memory at the end; for launches that leave SMs to spare, where the
+// chain of rounds of a single warp is what the call waits for.
+template <int SPLIT>
+__global__ void __launch_bounds__(kSmallMaxWarps * 32 * SPLIT) fwd_small_kernel(FwdParams p, SmallLists lists) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q_rows = ((p.n_k + 15) >> 4) * 16;  // 16 per computing warp; further warps only help staging
@@ -73,6 +79,7 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
   uint16_t* Ks = Qs + q_rows * kRowPad;                   // [l_pad][kRowPad]
   uint16_t* Vs = Ks + l_pad * kRowPad;                    // [l_pad][kRowPad]
   uint32_t* Ms = reinterpret_cast<uint32_t*>(Vs + l_pad * kRowPad);  // [q_rows][8]: live bits of keys 0 .. 255
+  float* Xs = reinterpret_cast<float*>(Ms + q_rows * 8);             // SPLIT 2: [q_rows / 16][kMergeFloats]
 
   asm volatile("griddepcontrol.launch_dependents;");
   const int h = blockIdx.x % p.n_heads, b = blockIdx.x / p.n_heads;
@@ -146,7 +153,8 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
   }
   __syncthreads();
 
-  const int row0 = warp * 16;
+  const int group = warp / SPLIT, part = warp % SPLIT;  // row group; which rounds of it this warp takes
+  const int row0 = group * 16;
   if (row0 >= n_k) {  // a warp without query rows only helped staging
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
@@ -170,7 +178,7 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
   const int shift = (lane & 3) * 2;  // element (j, e) of a row is key 64 kb + 8 j + 2 (lane % 4) + e
   constexpr uint32_t kOnes = 0x3f803f80u;  // bf16 pair (1, 1)
 
-  for (int kb = 0; kb < n64; ++kb) {  // 64 keys per round
+  for (int kb = part; kb < n64; kb += SPLIT) {  // 64 keys per round
     const uint32_t wl[2] = {m_lo[kb * 2], m_lo[kb * 2 + 1]};
     const uint32_t wh[2] = {m_hi[kb * 2], m_hi[kb * 2 + 1]};
     // 16-key groups with no live key in any of the warp's 16 rows are skipped (also the padding past L_k)
@@ -266,6 +274,47 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
     __syncthreads();
   }
 
+  if (SPLIT == 2) {
+    // ---- the pair's second warp hands its partial result (running maximum, row sum, unnormalised output)
+    // to the first, which rescales both to the common maximum
+    float* Xo = Xs + group * kMergeFloats;
+    float* Xm = Xo + 16 * kMergePad;
+    float* Xl = Xm + 16;
+    const int r_lo = lane >> 2, cq = (lane & 3) * 2;
+    if (part == 1) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        *reinterpret_cast<float2*>(Xo + r_lo * kMergePad + j * 8 + cq) = make_float2(o[j][0], o[j][1]);
+        *reinterpret_cast<float2*>(Xo + (r_lo + 8) * kMergePad + j * 8 + cq) = make_float2(o[j][2], o[j][3]);
+      }
+      if ((lane & 3) == 0) {
+        Xm[r_lo] = m_run[0];
+        Xm[r_lo + 8] = m_run[1];
+        Xl[r_lo] = lsum[0];
+        Xl[r_lo + 8] = lsum[2];
+      }
+      __threadfence_block();
+      asm volatile("bar.arrive %0, 64;" ::"r"(1 + group) : "memory");
+      return;
+    }
+    asm volatile("bar.sync %0, 64;" ::"r"(1 + group) : "memory");
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      const int row = r_lo + 8 * x;
+      const float m1 = Xm[row], l1 = Xl[row];
+      const float m_new = fmaxf(m_run[x], m1);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float a0 = ex2(m_run[x] - m_use), a1 = ex2(m1 - m_use);
+      lsum[2 * x] = lsum[2 * x] * a0 + l1 * a1;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float2 o1 = *reinterpret_cast<const float2*>(Xo + row * kMergePad + j * 8 + cq);
+        o[j][2 * x] = o[j][2 * x] * a0 + o1.x * a1;
+        o[j][2 * x + 1] = o[j][2 * x + 1] * a0 + o1.y * a1;
+      }
+    }
+  }
+
   // ---- normalise, gather the warp's 16 rows in its (now free) Q rows, store 16 bytes per lane
   const float inv[2] = {1.f / lsum[0], 1.f / lsum[2]};
   __syncwarp();
@@ -294,44 +343,55 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32) fwd_small_kernel(FwdParam
 
 }  // namespace
 
-bool small_step_eligible(int n_q_tiles, int n_key_tiles, bool raster_only, int n_k, int L_k) {
-  if (!raster_only || n_q_tiles != 1 || n_key_tiles < 1 || n_key_tiles > 2) return false;
-  // Legacy warp-level mma is several times slower than tcgen05 on this part, so the kernel only wins while
-  // the step is latency-bound: up to 18 (16-row warp) x (64-key round) units of work per CTA.  Measured on
-  // B200 with 128, 288 and 960 (batch row, head) units: 64 x 155 and 81 x 147 steps are faster here,
-  // the 100 x 255 step is faster on the tcgen05 kernel.
-  const int warps = (n_k + 15) / 16, rounds = (L_k + 63) / 64;
-  return warps * rounds <= 18;
+bool small_step_candidate(int n_q_tiles, int n_key_tiles, bool raster_only) {
+  return raster_only && n_q_tiles == 1 && n_key_tiles >= 1 && n_key_tiles <= 2;
 }
 
-cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, cudaStream_t stream) {
+int small_step_mode(int n_k, int L_k, long long units, int n_sm) {
+  const int warps = (n_k + 15) / 16, rounds = (L_k + 63) / 64;
+  // Legacy warp-level mma is several times slower than tcgen05 on this part, so the kernel only wins while
+  // the step is a latency chain: up to 18 (16-row warp) x (64-key round) units of work per CTA.  Measured on
+  // B200 with 128, 288 and 960 (batch row, head) units: 64 x 155 and 81 x 147 steps are faster here, the
+  // 100 x 255 step is faster on the tcgen05 kernel (8.4 against 8.9 us even with two warps per row group).
+  if (warps * rounds > 18) return 0;
+  // A launch that leaves SMs to spare waits for the chain of rounds of single warps: two warps per row group
+  // as soon as there is more than one round (4.8 -> 4.4 us at 36 x 91, 6.9 -> 6.1 us at 64 x 155, 128 units).
+  return units <= n_sm && rounds >= 2 ? 2 : 1;
+}
+
+template <int SPLIT>
+static cudaError_t launch_small_variant(const FwdParams& p, const SmallLists& lists, int n_sm, cudaStream_t stream) {
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
-  constexpr int kMaxSmem = (kBlockM + 2 * 2 * kBlockN) * kRowPad * 2 + kBlockM * 32;
+  constexpr int kMaxSmem = (kBlockM + 2 * 2 * kBlockN) * kRowPad * 2 + kBlockM * 32 +
+                           (SPLIT == 2 ? (kBlockM / 16) * kMergeFloats * 4 : 0);
   std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(fwd_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    attr_err = cudaFuncSetAttribute(fwd_small_kernel<SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
   });
   if (attr_err != cudaSuccess) return attr_err;
   const int q_rows = (p.n_k + 15) / 16 * 16, l_pad = (p.L_k + 15) & ~15;
-  // one warp per 16 query rows; more where the staging copies would otherwise queue up behind few threads,
+  // SPLIT warps per 16 query rows; more where the staging copies would otherwise queue up behind few threads,
   // unless the grid fills the SMs several times over (idle warps still hold registers and cost residency)
-  int n_warps = q_rows / 16;
-  int dev = 0, n_sm = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess) (void)cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  int n_warps = q_rows / 16 * SPLIT;
   const int stage_warps = ((q_rows + 2 * l_pad) * 8 + 191) / 192;
   if (n_warps < stage_warps && (long long)p.n_heads * p.batch_computed <= 2LL * n_sm)
-    n_warps = stage_warps < kSmallMaxWarps ? stage_warps : kSmallMaxWarps;
+    n_warps = stage_warps < kSmallMaxWarps * SPLIT ? stage_warps : kSmallMaxWarps * SPLIT;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)p.n_heads * (unsigned)p.batch_computed);
   cfg.blockDim = dim3((unsigned)n_warps * 32);
-  cfg.dynamicSmemBytes = (size_t)(q_rows + 2 * l_pad) * kRowPad * 2 + (size_t)q_rows * 32;
+  cfg.dynamicSmemBytes = (size_t)(q_rows + 2 * l_pad) * kRowPad * 2 + (size_t)q_rows * 32 +
+                         (SPLIT == 2 ? (size_t)(q_rows / 16) * kMergeFloats * 4 : 0);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = p.overlap_launch ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, fwd_small_kernel, p, lists);
+  return cudaLaunchKernelEx(&cfg, fwd_small_kernel<SPLIT>, p, lists);
+}
+
+cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, int mode, int n_sm, cudaStream_t stream) {
+  return mode == 2 ? launch_small_variant<2>(p, lists, n_sm, stream) : launch_small_variant<1>(p, lists, n_sm, stream);
 }
 
 }  // namespace litevar

@@ -117,10 +117,13 @@ struct FwdParams {
 
 cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
 
-// Small steps (one query tile, at most two raster key tiles, little enough work): warp-level mma on a shared-memory copy of the
-// whole K/V prefix.  `lists` is set 0's tile list (per-head sets are looked up on the device).
-bool small_step_eligible(int n_q_tiles, int n_key_tiles, bool raster_only, int n_k, int L_k);
-cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, cudaStream_t stream);
+// Small steps (one query tile, at most two raster key tiles): warp-level mma on a shared-memory copy of the whole
+// K/V prefix.  `small_step_candidate` is the plan-time test; `small_step_mode` decides per launch from the
+// work and the number of (batch row, head) units: 0 = use the tcgen05 kernel, 1 = one warp per 16 query rows, 2 = two.
+// `lists` is set 0's tile list (per-head sets are looked up on the device).
+bool small_step_candidate(int n_q_tiles, int n_key_tiles, bool raster_only);
+int small_step_mode(int n_k, int L_k, long long units, int n_sm);
+cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, int mode, int n_sm, cudaStream_t stream);
 
 // Tensor-core path.  Returns LITEVAR_OK or an error status (tensor-map encoding can fail).
 litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
@@ -132,7 +135,7 @@ struct litevar_plan {
   int32_t n_heads = 0, n_sets = 1, shape = 0, n_global = 0, rho_num = 1, rho_den = 4, tiling = 0;
   float sm_scale = 0.125f;
   int32_t kernel = LITEVAR_KERNEL_AUTO;
-  int device = 0;
+  int device = 0, n_sm = 148;
   std::vector<int32_t> radius;        // [n_sets][K][K]
   std::vector<int32_t> head_to_set;   // [H] (empty when n_sets == 1)
   int32_t* d_head_to_set = nullptr;

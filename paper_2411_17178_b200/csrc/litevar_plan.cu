@@ -425,15 +425,12 @@ bool strides_ok(const litevar_strides_t* s) {
          (s->head % 8) == 0 && (s->token % 8) == 0;
 }
 
-// The kernel a forward of this step launches under the plan's current selection.
-int32_t step_kernel(const litevar_plan_t* plan, const Step& st) {
-  if (plan->kernel == LITEVAR_KERNEL_SIMT) return LITEVAR_KERNEL_SIMT;
-  if (plan->kernel == LITEVAR_KERNEL_AUTO) {
-    bool all_small = true;  // every window set of the step has a list the small-step kernel can take
-    for (const StepSet& ss : st.sets) all_small = all_small && ss.small.n > 0;
-    if (all_small) return LITEVAR_KERNEL_SMALL;
-  }
-  return LITEVAR_KERNEL_TCGEN05;
+// How the small-step kernel would run this step for `units` (batch row, head) units: 0 = not at all.
+int small_mode(const litevar_plan_t* plan, const Step& st, long long units) {
+  if (plan->kernel != LITEVAR_KERNEL_AUTO) return 0;
+  for (const StepSet& ss : st.sets)  // every window set of the step has a list the small-step kernel can take
+    if (ss.small.n <= 0) return 0;
+  return small_step_mode(st.n_k, st.L_k, units, plan->n_sm);
 }
 
 }  // namespace
@@ -488,6 +485,7 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
   if (!plan) return LITEVAR_ERR_OOM;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   plan->device = dev;
+  plan->n_sm = prop.multiProcessorCount;
   plan->n_heads = n_heads;
   plan->n_sets = window->n_sets;
   plan->shape = window->shape;
@@ -592,7 +590,7 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
       if ((s = plan_step_set(plan, k0, set, stream)) != LITEVAR_OK) return fail(s);
       descs[set] = SetDesc{st.sets[set].d_row_ptr, st.sets[set].d_pairs, st.sets[set].d_mask};
       StepSet& ss = st.sets[set];
-      if (small_step_eligible(st.n_q_tiles, st.n_key_tiles, !st.q_patch && st.first_patch == k0 + 1, st.n_k, st.L_k) &&
+      if (small_step_candidate(st.n_q_tiles, st.n_key_tiles, !st.q_patch && st.first_patch == k0 + 1) &&
           ss.n_pairs >= 1 && ss.n_pairs <= 2) {
         ss.small.n = ss.n_pairs;
         if (cudaMemcpyAsync(ss.small.pr, ss.d_pairs, sizeof(Pair) * ss.n_pairs, cudaMemcpyDeviceToHost, stream) !=
@@ -656,8 +654,8 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   for (const StepSet& ss : st.sets) p.first_tile_zero &= ss.first_tile_zero ? 1 : 0;
   p.pairs_per_tile = (st.sets[0].n_pairs + st.n_q_tiles - 1) / st.n_q_tiles;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (step_kernel(plan, st) == LITEVAR_KERNEL_SMALL) {
-    if (launch_forward_small(p, st.sets[0].small, stream) != cudaSuccess) {
+  if (const int mode = small_mode(plan, st, (long long)p.n_heads * p.batch_computed)) {
+    if (launch_forward_small(p, st.sets[0].small, mode, plan->n_sm, stream) != cudaSuccess) {
       (void)cudaGetLastError();
       return LITEVAR_ERR_CUDA;
     }
@@ -793,9 +791,14 @@ litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel) {
   return LITEVAR_OK;
 }
 
-litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t* kernel) {
-  if (!plan || !kernel || step_k < 1 || step_k > plan->sched.n_scales) return LITEVAR_ERR_INVALID_ARG;
-  *kernel = step_kernel(plan, plan->steps[step_k - 1]);
+litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
+                                          int32_t* kernel) {
+  if (!plan || !kernel || step_k < 1 || step_k > plan->sched.n_scales || batch_pairs < 1) return LITEVAR_ERR_INVALID_ARG;
+  const Step& st = plan->steps[step_k - 1];
+  const long long units = (long long)plan->n_heads * (st.share ? batch_pairs : 2 * batch_pairs);
+  *kernel = plan->kernel == LITEVAR_KERNEL_SIMT ? LITEVAR_KERNEL_SIMT
+            : small_mode(plan, st, units)       ? LITEVAR_KERNEL_SMALL
+                                                : LITEVAR_KERNEL_TCGEN05;
   return LITEVAR_OK;
 }
 

@@ -70,6 +70,6 @@ def test_plan_argument_validation_before_device_work(lib):
 def test_null_plan_calls(lib):
     assert lib.litevar_plan_poll_device_status(None) == 1
     assert lib.litevar_plan_set_kernel(None, 0) == 1
-    assert lib.litevar_plan_step_kernel(None, 1, None) == 1
+    assert lib.litevar_plan_step_kernel(None, 1, 1, None) == 1
     assert lib.litevar_plan_stats(None, 1, 0, None, None, None, None) == 1
     lib.litevar_plan_destroy(None)

@@ -308,18 +308,20 @@ def test_bench_launch_configuration_sampled(cfg, steps):
 
 def test_step_kernel_selection():
     """AUTO runs the small-step kernel on steps with one query tile, at most two raster key tiles and little
-    work, the tcgen05 kernel elsewhere; forcing a kernel or patch tiles overrides it."""
+    work, whatever the batch; the tcgen05 kernel elsewhere; forcing a kernel or patch tiles overrides it."""
     lib_ready()
     S, T, M = binding.KERNEL_SIMT, binding.KERNEL_TCGEN05, binding.KERNEL_SMALL
     plan = binding.Plan(wl.SCALES_256, n_heads=2)
-    assert [plan.step_kernel(k) for k in range(1, 11)] == [M] * 7 + [T] * 3
+    assert [plan.step_kernel(k, 1) for k in range(1, 11)] == [M] * 7 + [T] * 3     # up to 64 x 155
+    assert [plan.step_kernel(k, 64) for k in range(1, 11)] == [M] * 7 + [T] * 3
     plan.set_kernel(T)
     assert [plan.step_kernel(k) for k in range(1, 11)] == [T] * 10
     plan.set_kernel(S)
     assert [plan.step_kernel(k) for k in range(1, 11)] == [S] * 10
     plan.close()
     plan = binding.Plan(wl.SCALES_512, n_heads=2)
-    assert [plan.step_kernel(k) for k in range(1, 11)] == [M] * 6 + [T] * 4
+    assert [plan.step_kernel(k, 1) for k in range(1, 11)] == [M] * 6 + [T] * 4     # step 7 has two query tiles
+    assert [plan.step_kernel(k, 64) for k in range(1, 11)] == [M] * 6 + [T] * 4
     plan.close()
     plan = binding.Plan(wl.SCALES_256, n_heads=2, tiling=binding.TILING_PATCH)
     assert [plan.step_kernel(k) for k in range(1, 11)] == [T] * 10   # patch query tiles at every step
@@ -337,7 +339,8 @@ def test_step_kernel_selection():
 ])
 def test_small_step_kernel_shape_extremes(scales, n_global, share):
     """Shapes at the edges of what the small-step kernel takes (row groups and key rounds with ragged ends,
-    the largest eligible warp x round products), each step checked in full against the oracle."""
+    one to four 64-key rounds shared by the two warps of a row group), each step checked in full against the
+    oracle."""
     lib_ready()
     H, B = 3, 1
     w = wl.small_workload(scales, n_heads=H, batch_pairs=B, share_cfg=share, index=90)
@@ -348,7 +351,7 @@ def test_small_step_kernel_shape_extremes(scales, n_global, share):
     for k in range(1, len(scales) + 1):
         n_k, L_k = orc.map_shape(scales, k)
         small = n_k <= 128 and L_k <= 256 and -(-n_k // 16) * -(-L_k // 64) <= 18
-        assert plan.step_kernel(k) == (binding.KERNEL_SMALL if small else binding.KERNEL_TCGEN05), (scales, k)
+        assert plan.step_kernel(k, B) == (binding.KERNEL_SMALL if small else binding.KERNEL_TCGEN05), (scales, k)
         assert small or k < len(scales)     # the step each case is about runs on the small-step kernel
         assert np.array_equal(plan.materialize_mask(k), orc.mask(scales, k, tab[k - 1]))
         Q = wl.make_q(w, 0, k)
