@@ -4,7 +4,9 @@
  * One operation: the attention that a VAR image generator runs at every coarse-to-fine
  * scale step (the current scale's queries against the K/V cache of all scales so far),
  * under LiteVAR's multi-diagonal window mask (MDWA, paper Section 2) and with LiteVAR's
- * attention sharing across classifier-free guidance (ASC, paper Section 3).
+ * attention sharing across classifier-free guidance (ASC, paper Section 3).  Beside it: the
+ * window calibration of Section 2 on saved attention maps (litevar_calibrate_windows) and the
+ * dynamic 8-bit quantiser of Q, K and V of Section 4 (litevar_quantize_rows, litevar_quantize_qkv).
  *
  * Notation (paper Section 2).  Scales s_1..s_K; scale k holds n_k = s_k^2 tokens in
  * row-major order of its s_k x s_k grid; off_j = sum_{i<j} n_i; L_k = sum_{i<=k} n_i.
