@@ -2,6 +2,7 @@
 """Benchmark of the LiteVAR attention path (multi-diagonal window mask + CFG sharing) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference] [--no-extras]
+                    [--kernel-only] [--calibration] [--dense] [--rho NUM DEN]
 
 A "step" is one pass of the whole hot path over one batch: one full generation's attention,
 i.e. every scale step of every layer of the chosen workload (for the single-call workloads 1 and
@@ -13,10 +14,15 @@ value            useful TFLOP/s: 256 FLOP per live map entry of every (batch row
                  the generation's calls replayed from one CUDA graph
 e2e              the same metric through the per-call API with pinned HOST buffers: every call
                  copies its Q and the new scale's K/V rows to the device and its output back
-roofline         HBM bound for this workload: compulsory bytes (Q + K/V prefix read once per
-                 computed (b, h), output written for all 2B rows) over the measured time
+roofline         HBM bound of the kernel that takes most of the generation (the steps it serves are
+                 replayed as a graph of their own and timed with CUDA events): compulsory bytes (Q +
+                 K/V prefix read once per computed (b, h), output written for all 2B rows) over that
+                 time; the other forward kernel is listed beside it
 cpu_baseline     the CPU fp64 oracle timed on this machine's host cores on a bounded sample
 all_configs      the five benchmark workloads, window and full-mask variants (unless --no-extras)
+calibration      the window calibration kernel against the HBM roofline (also: --calibration alone)
+qkv8             the 8-bit Q/K/V row quantiser against the HBM roofline, and the headline generation
+                 with Q and the appended K/V rows quantised before every call
 
 With --impl reference the oracle itself is timed (rank 0 only) and printed in the same format.
 """
