@@ -128,6 +128,15 @@ def _stream_ptr(stream) -> Optional[int]:
     return getattr(stream, "cuda_stream", stream)
 
 
+def _current_raw_stream(device_index) -> int:
+    """cudaStream_t of torch's current stream on that device, without building a Stream object."""
+    import torch
+    try:
+        return torch._C._cuda_getCurrentRawStream(device_index if device_index is not None else torch.cuda.current_device())
+    except AttributeError:
+        return torch.cuda.current_stream().cuda_stream
+
+
 def _strides(t) -> _Strides:
     assert t.dim() == 4 and t.stride(3) == 1, "expected [2B, H, tokens, 64] with contiguous head_dim"
     return _Strides(t.stride(0), t.stride(1), t.stride(2))
@@ -170,6 +179,8 @@ class Plan:
                                    ctypes.byref(handle))
         _check(st, "litevar_attn_plan")
         self._h = handle
+        self._strides4 = tuple(_Strides(0, 0, 0) for _ in range(4))
+        self._strides4_ref = tuple(ctypes.byref(x) for x in self._strides4)
 
     def close(self) -> None:
         if getattr(self, "_h", None):
@@ -184,13 +195,30 @@ class Plan:
 
     # -- forward ---------------------------------------------------------------------------
     def forward(self, step_k: int, batch_pairs: int, q, k_cache, v_cache, out, stream=None) -> None:
-        """litevar_attn_forward on torch CUDA tensors (bf16, [2B, H, tokens, 64])."""
-        st = self._lib.litevar_attn_forward(
-            self._h, int(step_k), int(batch_pairs),
-            q.data_ptr(), ctypes.byref(_strides(q)), k_cache.data_ptr(), ctypes.byref(_strides(k_cache)),
-            v_cache.data_ptr(), ctypes.byref(_strides(v_cache)), out.data_ptr(), ctypes.byref(_strides(out)),
-            _stream_ptr(stream))
-        _check(st, "litevar_attn_forward")
+        """litevar_attn_forward on torch CUDA tensors (bf16, [2B, H, tokens, 64]).
+
+        The marshalling is kept short (it is most of an eager call's host time): the four stride structs live
+        in the plan and are refilled, so one plan must not be driven from several Python threads at once."""
+        sq, sk, sv, so = self._strides4
+        a = q.stride()
+        sq.batch, sq.head, sq.token = a[0], a[1], a[2]
+        b = k_cache.stride()
+        sk.batch, sk.head, sk.token = b[0], b[1], b[2]
+        c = v_cache.stride()
+        sv.batch, sv.head, sv.token = c[0], c[1], c[2]
+        d = out.stride()
+        so.batch, so.head, so.token = d[0], d[1], d[2]
+        if a[3] != 1 or b[3] != 1 or c[3] != 1 or d[3] != 1:
+            raise ValueError("expected [2B, H, tokens, 64] tensors with contiguous head_dim")
+        if stream is None:
+            stream_ptr = _current_raw_stream(q.device.index)
+        else:
+            stream_ptr = getattr(stream, "cuda_stream", stream)
+        st = self._lib.litevar_attn_forward(self._h, step_k, batch_pairs, q.data_ptr(), self._strides4_ref[0],
+                                            k_cache.data_ptr(), self._strides4_ref[1], v_cache.data_ptr(),
+                                            self._strides4_ref[2], out.data_ptr(), self._strides4_ref[3], stream_ptr)
+        if st != 0:
+            _check(st, "litevar_attn_forward")
 
     def forward_raw(self, step_k, batch_pairs, q_ptr, q_str, k_ptr, k_str, v_ptr, v_str, o_ptr, o_str,
                     stream_ptr) -> int:

@@ -821,8 +821,7 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
   if (!ok) return LITEVAR_ERR_INVALID_ARG;
   // A step with a single query tile and more CTAs than SMs runs the small build: two CTAs share an SM and
   // hide each other's set-up and drain.  With fewer CTAs than SMs sharing would only halve each CTA's SM.
-  int dev = 0, n_sm = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess) (void)cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  const int n_sm = current_sm_count();
   const long long units = (long long)p.n_heads * p.batch_computed;
   // ... and so does a step whose lists are short (set-up and drain weigh more than the shared K/V staging saves)
   const bool lite = (n_q_tiles == 1 && units > n_sm) ||

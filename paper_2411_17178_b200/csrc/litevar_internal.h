@@ -115,6 +115,19 @@ struct FwdParams {
                                 // stream has finished (the plan it reads was complete long before)
 };
 
+// SM count of the current device, looked up once per device (the attribute query costs a microsecond).
+inline int current_sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  int n = cached[dev];
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    cached[dev] = n;  // benign race: every writer stores the same value
+  }
+  return n;
+}
+
 cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
 
 // Small steps (one query tile, at most two raster key tiles): warp-level mma on a shared-memory copy of the whole
