@@ -184,7 +184,7 @@ litevar_status_t litevar_attn_forward_static(const int32_t* scales, int32_t n_sc
  * taken over all given maps and query rows) reaches the threshold R_0.  Square windows only.
  *
  *   maps     device float32 [n_maps][n_k][L_k], contiguous, non-negative (rows need not sum to 1)
- *   r0       threshold R_0 in (0, 1]; the decision is window mass >= (double)r0 * part mass in fp64
+ *   r0       threshold R_0 in (0, 1]; the decision is window mass >= r0 * part mass in fp64
  *   radius   host out [n_scales]: -1 for parts j <= n_global_scales and for j > step_k, else the radius;
  *            a row of this kind is what litevar_window_t.radius takes
  *   ratio    host out [n_scales][256] or NULL: R_w for w = 0 .. s_j - 1 (1 elsewhere)
@@ -193,7 +193,7 @@ litevar_status_t litevar_attn_forward_static(const int32_t* scales, int32_t n_sc
  * Errors: INVALID_ARG, OOM, CUDA.
  */
 litevar_status_t litevar_calibrate_windows(const int32_t* scales, int32_t n_scales, int32_t step_k,
-                                           int32_t n_global_scales, const float* maps, int64_t n_maps, float r0,
+                                           int32_t n_global_scales, const float* maps, int64_t n_maps, double r0,
                                            int32_t* radius, double* ratio, void* stream);
 
 /* Counts for step k and window set `set`: live map entries, live / full / partial tile pairs. */
@@ -252,8 +252,8 @@ litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t st
  * a bf16 tensor x[batch][n_heads][n_tokens][head_dim] (element strides sx, head_dim contiguous) to `bits`-bit
  * integers with a scale and a zero point taken from the row's maximum and minimum:
  *     z = (max + min) / 2,  s = (max - min) / (2^bits - 1),
- *     code = clamp(round((x - z) * r), -2^(bits-1), 2^(bits-1) - 1), r = 1 / s   (round to nearest even; s = 0:
- *     code 0), all in fp32, one IEEE operation at a time.  Outputs, each optional (NULL = not wanted), all device memory:
+ *     code = clamp(round((x - z) / s), -2^(bits-1), 2^(bits-1) - 1)   (round to nearest even; s = 0: code 0),
+ *     all in fp32, one correctly rounded IEEE operation at a time (the quotient is an IEEE division).  Outputs, each optional (NULL = not wanted), all device memory:
  *   x_dq   bf16, strides sdq: the dequantised rows code * s + z rounded to bf16 - what the attention then reads;
  *          may be x itself (in place)
  *   codes  int8 [batch][n_heads][n_tokens][head_dim], dense, 8-byte aligned

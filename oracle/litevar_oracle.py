@@ -251,7 +251,7 @@ def calibrate_radius(scales: Sequence[int], k: int, maps: np.ndarray, r0: float,
             w_row = [GLOBAL] * len(scales)
             w_row[j - 1] = w
             inside = (part * mask(scales, k, w_row)[None, :, off[j - 1]:off[j]]).sum()
-            if inside >= np.float64(np.float32(r0)) * total or w >= int(scales[j - 1]) - 1:
+            if inside >= np.float64(r0) * total or w >= int(scales[j - 1]) - 1:
                 break
             w += 1
         out[j - 1] = w
@@ -270,9 +270,9 @@ def quantize_rows(x: np.ndarray, bits: int = 8):
     """Dynamic min-max quantisation of Section 4, one (s, z) per row (last axis).
 
     The decision which integer a value becomes is taken in fp32, one IEEE operation at a time, in the
-    order written here: z = (max + min) * 0.5; s = (max - min) / (2^B - 1); r = 1 / s;
-    code = clamp(rint((x - z) * r), -2^(B-1), 2^(B-1) - 1); dequantised = bf16(code * s + z).
-    (The division by s is taken as a multiplication by the row's reciprocal step, one division per row.)
+    order written here: z = (max + min) * 0.5; s = (max - min) / (2^B - 1);
+    code = clamp(rint((x - z) / s), -2^(B-1), 2^(B-1) - 1); dequantised = bf16(code * s + z).
+    The quotient (x - z) / s is the division the section's formula prints, rounded once to fp32.
     A constant row (s = 0) has code 0 everywhere and dequantises to z.
     Returns (codes int32, s fp32 [..., 1], z fp32 [..., 1], dequantised fp32 holding bf16 values)."""
     x = np.asarray(x, dtype=np.float32)
@@ -281,8 +281,7 @@ def quantize_rows(x: np.ndarray, bits: int = 8):
     z = (mx + mn) * np.float32(0.5)
     s = (mx - mn) / np.float32(2 ** bits - 1)
     safe = np.where(s > 0, s, np.float32(1))
-    r = np.float32(1) / safe
-    code = np.rint((x - z) * r)
+    code = np.rint((x - z) / safe)
     code = np.clip(code, -(2 ** (bits - 1)), 2 ** (bits - 1) - 1)
     code = np.where(s > 0, code, np.float32(0)).astype(np.float32)
     deq = round_to_bf16((code * s).astype(np.float32) + z)

@@ -80,7 +80,7 @@ def load() -> ctypes.CDLL:
                                                 P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides),
                                                 P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides), P]
     lib.litevar_calibrate_windows.restype = ctypes.c_int
-    lib.litevar_calibrate_windows.argtypes = [ctypes.POINTER(I32), I32, I32, I32, P, I64, ctypes.c_float, P, P, P]
+    lib.litevar_calibrate_windows.argtypes = [ctypes.POINTER(I32), I32, I32, I32, P, I64, ctypes.c_double, P, P, P]
     lib.litevar_quantize_rows.restype = ctypes.c_int
     lib.litevar_quantize_rows.argtypes = [P, ctypes.POINTER(_Strides), I32, I32, I32, I32, I32, P,
                                           ctypes.POINTER(_Strides), P, P, P, P]

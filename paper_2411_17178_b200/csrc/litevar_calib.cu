@@ -186,10 +186,10 @@ using namespace litevar;
 
 extern "C" litevar_status_t litevar_calibrate_windows(const int32_t* scales, int32_t n_scales, int32_t step_k,
                                                       int32_t n_global_scales, const float* maps, int64_t n_maps,
-                                                      float r0, int32_t* radius, double* ratio, void* stream_) {
+                                                      double r0, int32_t* radius, double* ratio, void* stream_) {
   if (!scales || !maps || !radius) return LITEVAR_ERR_INVALID_ARG;
   if (n_scales < 1 || n_scales > kMaxScales || step_k < 1 || step_k > n_scales || n_maps < 1 ||
-      n_global_scales < 0 || !(r0 > 0.f) || r0 > 1.f)
+      n_global_scales < 0 || !(r0 > 0.0) || r0 > 1.0)
     return LITEVAR_ERR_INVALID_ARG;
   for (int i = 0; i < n_scales; ++i)
     if (scales[i] < 1 || scales[i] > kMaxScale) return LITEVAR_ERR_INVALID_ARG;
@@ -273,7 +273,7 @@ extern "C" litevar_status_t litevar_calibrate_windows(const int32_t* scales, int
     for (int d = 0; d < scales[j]; ++d) {
       cum += h[d];
       if (ratio) ratio[(size_t)j * kMaxDist + d] = total > 0.0 ? cum / total : 1.0;
-      if (!found && cum >= (double)r0 * total) {
+      if (!found && cum >= r0 * total) {
         w = d;
         found = true;
       }

@@ -1,7 +1,10 @@
 // Dynamic min-max quantisation of Q, K or V rows to B-bit integers (paper Section 4, "QKV8"): for every token
 // row of a head (64 values) z = (max + min) / 2, s = (max - min) / (2^B - 1),
-// code = clamp(round((x - z) / s), -2^(B-1), 2^(B-1) - 1), and the attention runs on code * s + z.  The division
-// by s is a multiplication by the row's reciprocal step r = 1 / s (one division per row).
+// code = clamp(round((x - z) / s), -2^(B-1), 2^(B-1) - 1), and the attention runs on code * s + z.  The code is
+// the one the correctly rounded fp32 quotient (x - z) / s gives: the quotient is first estimated as
+// (x - z) * (1 / s), which is within two units in the last place of it; only an estimate that close to a
+// rounding tie (a half-integer) can round to another integer than the quotient does, and those few elements
+// take the IEEE division.
 //
 // In a generation the rows of a step are quantised once, when they are appended to the K/V cache (and Q as it
 // is produced); the attention kernels then read the dequantised bf16 rows unchanged.  The pass is bound by
@@ -98,7 +101,8 @@ __global__ void __launch_bounds__(kQuantThreads) quant_rows_kernel(QuantArgs a) 
     }
     const float z = __fmul_rn(__fadd_rn(mx, mn), 0.5f);
     const float s = __fdiv_rn(__fsub_rn(mx, mn), a.levels);
-    const float r = __fdiv_rn(1.f, s > 0.f ? s : 1.f);  // one division per row; the elements multiply
+    const float s1 = s > 0.f ? s : 1.f;
+    const float r = __fdiv_rn(1.f, s1);  // one division per row; the elements multiply, see below
     float c[8];
     uint32_t packed[4];
 #pragma unroll
@@ -107,8 +111,16 @@ __global__ void __launch_bounds__(kQuantThreads) quant_rows_kernel(QuantArgs a) 
       if (s > 0.f) {
         // round to nearest even without the conversion pipe: adding and subtracting 1.5 * 2^23 is exact
         // rounding to an integer for |y| < 2^22, and |y| stays near 2^(B-1) here
-        const float y = __fmul_rn(__fsub_rn(v[i], z), r);
-        q = fminf(fmaxf(__fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f), a.lo), a.hi);
+        const float d = __fsub_rn(v[i], z);
+        float y = __fmul_rn(d, r);
+        float n = __fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f);
+        // |y| <= 2^(B-1) + 1, so two units in the last place are at most 2^-14: an estimate farther than
+        // 2^-12 from a half-integer rounds as the exact quotient does
+        if (fabsf(__fsub_rn(y, n)) > 0.5f - 0.000244140625f) {
+          y = __fdiv_rn(d, s1);
+          n = __fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f);
+        }
+        q = fminf(fmaxf(n, a.lo), a.hi);
       }
       c[i] = q;
     }

@@ -325,9 +325,9 @@ def test_calibration_monotone_and_limits():
             assert (rad[3:k] >= prev[3:k]).all()              # a stricter threshold never shrinks a window
         for j in range(4, k + 1):                             # smallest radius that reaches the threshold
             w = int(rad[j - 1])
-            assert orc.window_ratio(scales, k, j, w, maps) >= np.float32(r0) - 1e-15
+            assert orc.window_ratio(scales, k, j, w, maps) >= r0 - 1e-15
             if w > 0:
-                assert orc.window_ratio(scales, k, j, w - 1, maps) < np.float32(r0)
+                assert orc.window_ratio(scales, k, j, w - 1, maps) < r0
         prev = rad
     # R_0 = 1 on strictly positive maps: full attention (Section 2), radius = the smallest that covers the part
     full = orc.calibrate_radius(scales, k, maps, 1.0)
@@ -514,6 +514,64 @@ def test_quantizer_hand_worked_row_with_ties():
     # dequantised = code + 127.5, which lies half-way between two bf16 values from 128 on (bf16 spacing 1)
     assert deq[0, :4].tolist() == [-0.5, 1.5, 1.5, 3.5]
     assert deq[0, 255] == 254.0 and deq[0, 254] == 254.0
+
+
+def _rational_to_fp32(y):
+    """Nearest fp32 (ties to even) of an exact rational, by integer arithmetic only (normal range)."""
+    from fractions import Fraction
+    if y == 0:
+        return Fraction(0)
+    sign, a = (-1 if y < 0 else 1), abs(y)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    assert Fraction(2) ** e <= a < Fraction(2) ** (e + 1) and -126 <= e <= 127
+    ulp = Fraction(2) ** (e - 23)
+    m = a / ulp                                    # in [2^23, 2^24)
+    f = m.numerator // m.denominator
+    rem = m - f
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and f % 2 == 1):
+        f += 1
+    return sign * f * ulp
+
+
+def _rint_even(y):
+    from fractions import Fraction
+    f = y.numerator // y.denominator               # floor
+    rem = y - f
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and f % 2 != 0):
+        f += 1
+    return int(f)
+
+
+def test_quantizer_divides_by_the_step_as_section_4_prints():
+    # Section 4 prints (x - z) / s.  Multiplying by a rounded reciprocal 1 / s instead lands on the other side
+    # of a cell boundary for a small fraction of the elements; this pin holds the oracle to the division.  A
+    # seeded search finds elements where the two forms give different codes; the expected code comes from
+    # exact rational arithmetic on the fp32 values of x - z and s: the quotient rounded once to fp32 (ties to
+    # even), then to the nearest integer (ties to even), then clamped.
+    from fractions import Fraction
+    rng = np.random.default_rng(20241117)
+    x = torch.from_numpy(rng.standard_normal((60000, 64)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    mx, mn = x.max(-1, keepdims=True), x.min(-1, keepdims=True)
+    z = (mx + mn) * np.float32(0.5)
+    s = (mx - mn) / np.float32(255)
+    d = x - z
+    by_div = np.clip(np.rint(d / s), -128, 127)
+    by_mul = np.clip(np.rint(d * (np.float32(1) / s)), -128, 127)
+    rows, cols = np.nonzero(by_div != by_mul)
+    assert len(rows) >= 20, "the search must find elements that tell the two forms apart"
+    code = orc.quantize_rows(x)[0]
+    for r, c in list(zip(rows, cols))[:200]:
+        q = _rational_to_fp32(Fraction(float(d[r, c])) / Fraction(float(s[r, 0])))
+        want = max(-128, min(127, _rint_even(q)))
+        assert want == int(by_div[r, c]) and want != int(by_mul[r, c])
+        assert int(code[r, c]) == want, (r, c, int(code[r, c]), want)
+    # the helper itself: exactly representable values, a tie that goes to the even mantissa, one that goes up
+    assert _rational_to_fp32(Fraction(3, 8)) == Fraction(3, 8)
+    assert _rational_to_fp32(Fraction(2 ** 24 + 1)) == Fraction(2 ** 24)
+    assert _rational_to_fp32(Fraction(2 ** 24 + 3)) == Fraction(2 ** 24 + 4)
+    assert _rational_to_fp32(Fraction(1, 3)) == Fraction(float(np.float32(1) / np.float32(3)))
 
 
 def test_quantizer_is_the_textbook_mid_rise_quantiser_between_ties():
