@@ -86,8 +86,9 @@ enum {
   LITEVAR_KERNEL_AUTO = 0,    /* per step: the small-step kernel where the step fits it, else the tcgen05 kernel */
   LITEVAR_KERNEL_SIMT = 1,    /* plain CUDA-core kernel (slow; cross-check and bring-up) */
   LITEVAR_KERNEL_TCGEN05 = 2, /* tcgen05/TMEM/TMA kernel for every step */
-  LITEVAR_KERNEL_SMALL = 3    /* reported by litevar_plan_step_kernel only: warp-level mma kernel for steps with one
+  LITEVAR_KERNEL_SMALL = 3,   /* reported by litevar_plan_step_kernel only: warp-level mma kernel for steps with one
                                  query tile, at most two raster key tiles and little work */
+  LITEVAR_KERNEL_TCGEN05_WS = 4 /* tcgen05 kernel with one softmax thread per query row, for every step */
 };
 
 /*

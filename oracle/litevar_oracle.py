@@ -354,11 +354,13 @@ def attention_step(scales: Sequence[int], k: int, w_row: Sequence[int], Q, Kc, V
 
 def attention_sampled(scales: Sequence[int], k: int, w_row: Sequence[int], Q, Kc, Vc,
                       samples: Sequence[Tuple[int, int, int]], sm_scale: Optional[float] = None,
-                      share_cfg: bool = False) -> np.ndarray:
+                      share_cfg: bool = False, band: bool = False) -> np.ndarray:
     """Outputs for selected (batch row, head, query) triples only: [len(samples), d] fp64.
 
     Used at sizes where evaluating every row is out of reach.  With share_cfg a sample in
     the unconditional half is computed from the conditional row b - B, as ASC defines it.
+    Samples of one (batch row, head) are evaluated together (one widening of that unit's K and V);
+    every row still goes through `mask` / `mask_band` and `attention_rows` as in `attention_step`.
     """
     n_k, L_k = map_shape(scales, k)
     rows = Q.shape[0]
@@ -367,11 +369,17 @@ def attention_sampled(scales: Sequence[int], k: int, w_row: Sequence[int], Q, Kc
         sm_scale = 1.0 / np.sqrt(d)
     B = rows // 2
     out = np.empty((len(samples), d), dtype=np.float64)
+    groups = {}
     for i, (b, h, q) in enumerate(samples):
         src = b - B if (share_cfg and b >= B) else b
-        lv = mask(scales, k, w_row, q_rows=[q])
-        out[i] = attention_rows(bf16_to_f64(Q[src, h, q:q + 1]), bf16_to_f64(Kc[src, h, :L_k]),
-                                bf16_to_f64(Vc[src, h, :L_k]), lv, sm_scale)[0]
+        groups.setdefault((src, h), []).append((i, q))
+    for (src, h), items in groups.items():
+        qs = [q for _, q in items]
+        lv = mask_band(scales, k, w_row, q_rows=qs) if band else mask(scales, k, w_row, q_rows=qs)
+        Qr = bf16_to_f64(Q[src, h])[qs]
+        res = attention_rows(Qr, bf16_to_f64(Kc[src, h, :L_k]), bf16_to_f64(Vc[src, h, :L_k]), lv, sm_scale)
+        for (i, _), row in zip(items, res):
+            out[i] = row
     return out
 
 

@@ -20,7 +20,7 @@ OK = 0
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "EMPTY_ROW", 4: "ARCH", 5: "OOM", 6: "CUDA",
                 7: "DEVICE_TIMEOUT"}
 WINDOW_SQUARE, WINDOW_BAND = 0, 1
-KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_SMALL = 0, 1, 2, 3
+KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_SMALL, KERNEL_TCGEN05_WS = 0, 1, 2, 3, 4
 TILING_AUTO, TILING_RASTER, TILING_PATCH = 0, 1, 2
 
 EXPORTS = (

@@ -12,8 +12,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblitevar.so")
-SOURCES = ["litevar_plan.cu", "litevar_fwd_simt.cu", "litevar_fwd_tc.cu", "litevar_fwd_small.cu", "litevar_static.cu", "litevar_calib.cu", "litevar_quant.cu"]
-HEADERS = [os.path.join(CSRC, "litevar_internal.h"), os.path.join(ROOT, "include", "litevar.h")]
+SOURCES = ["litevar_plan.cu", "litevar_fwd_simt.cu", "litevar_fwd_tc.cu", "litevar_fwd_ws.cu", "litevar_fwd_small.cu", "litevar_static.cu", "litevar_calib.cu", "litevar_quant.cu"]
+HEADERS = [os.path.join(CSRC, "litevar_internal.h"), os.path.join(CSRC, "litevar_tc_ptx.h"), os.path.join(ROOT, "include", "litevar.h")]
 
 
 def _nvcc() -> str:

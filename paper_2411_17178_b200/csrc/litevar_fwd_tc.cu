@@ -31,25 +31,20 @@
 //
 // Every wait is bounded: when a wait runs out the CTA raises the plan's status word, drains its
 // outstanding copies, frees its TMEM and returns.
-#include <cuda.h>
-#include <cuda_bf16.h>
-#include <cuda_runtime.h>
-
 #include <cstring>
 #include <mutex>
 
-#include "litevar_internal.h"
+#include "litevar_tc_ptx.h"
 
 namespace litevar {
 
+using namespace tc;
+
 namespace {
 
-constexpr uint32_t kTileBytes = kBlockN * kHeadDim * 2;  // 16 KB: 128 rows of 128 B
 constexpr uint32_t kColS = 0;                // S_h at 128 h; O_h behind the S blocks; P_h overlays S_h
 constexpr int kOutCols = kHeadDim + 16;      // V columns + the ones block (row sums)
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 constexpr float kRescaleThreshold = 8.f;  // log2 units
-constexpr int kNoTile = 0x7fffffff;
 constexpr uint32_t kSlotSpinLimit = 1u << 26;  // polls of a shared-memory word before a softmax thread gives up
 
 // Two builds of the kernel.  Full: two query tiles per CTA, four K/V stages, 640 threads, all 512 TMEM
@@ -86,234 +81,6 @@ constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(k
                               ((uint32_t)(kBlockM >> 4) << 24);
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) |
                               ((uint32_t)(kOutCols >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// Shared-memory matrix descriptor for a tile of 128-byte rows written by TMA with the 128-byte
-// swizzle: 8-row groups are 1024 B apart (stride byte offset); version 1; layout type 2 = SWIZZLE_128B.
-// The same encoding serves a K-major operand (Q, K: rows = M/N index, 64 contiguous K elements) and the
-// MN-major V operand (rows = keys = K index, 64 contiguous N elements).
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
-  return (uint64_t)((saddr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
-         (2ull << 61);
-}
-// MN-major operand wider than one 64-element block: the leading-dimension byte offset (bits 16-29)
-// is the distance from the first block of N columns to the next one.
-__device__ __forceinline__ uint64_t make_desc_mn(uint32_t saddr, uint32_t next_block_bytes) {
-  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((next_block_bytes >> 4) & 0x3FFFu) << 16) |
-         ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try(uint64_t* bar, uint32_t parity) {
-  uint32_t done;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(done)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return done;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false when another role gave up or the time limit passed; the caller then
-// leaves its loop and falls through to the common teardown.
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                            int32_t* status) {
-  const unsigned long long t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if ((it & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicExch(status, 1);
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status) {
-  if (mbar_try(bar, parity)) return true;
-  if (mbar_try(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status);
-}
-
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                            uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
-      : "memory");
-}
-
-__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
-                                            uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar))
-      : "memory");
-}
-// Tensor maps of one launch.  q is rank 4 (raster query tiles) or rank 5 (patch query tiles); kr/vr
-// cover the raster prefix of the cache; k2/v2[i] cover the grid of the i-th key scale tiled in patches.
-struct TensorMaps {
-  CUtensorMap q, kr, vr;
-  CUtensorMap k2[kMaxPatchScales], v2[kMaxPatchScales];
-};
-
-// Loads of one query / key tile according to its geometry.
-__device__ __forceinline__ void load_q_tile(void* dst, const TensorMaps& tm, const FwdParams& p, int qt, int h, int b,
-                                            uint64_t* bar) {
-  if (p.q_geom == nullptr) {
-    tma_load_4d(dst, &tm.q, 0, qt * kBlockM, h, b, bar);
-    return;
-  }
-  const TileGeom g = p.q_geom[qt];
-  if (g.scale < 0)
-    tma_load_4d(dst, &tm.q, 0, g.a, h, b, bar);
-  else
-    tma_load_5d(dst, &tm.q, 0, g.b, g.a, h, b, bar);
-}
-__device__ __forceinline__ void load_kv_tile(void* dst, const CUtensorMap* raster, const CUtensorMap* patch,
-                                             const FwdParams& p, int kt, int h, int b, uint64_t* bar) {
-  if (p.key_geom == nullptr) {
-    tma_load_4d(dst, raster, 0, kt * kBlockN, h, b, bar);
-    return;
-  }
-  const TileGeom g = p.key_geom[kt];
-  if (g.scale < 0)
-    tma_load_4d(dst, raster, 0, g.a, h, b, bar);
-  else
-    tma_load_5d(dst, patch + g.map_slot, 0, g.b, g.a, h, b, bar);
-}
-
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-               : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t d;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-  return d;
-}
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-
-// Walk of the union of two ascending key-tile lists (the two halves of the CTA).
-struct UnionWalk {
-  const Pair* pairs;
-  int i0, e0, i1, e1;
-  int kt0, kt1;  // heads of the two lists (kNoTile when exhausted)
-  __device__ __forceinline__ void init(const Pair* p, int b0, int end0, int b1, int end1) {
-    pairs = p;
-    i0 = b0; e0 = end0; i1 = b1; e1 = end1;
-    kt0 = i0 < e0 ? __ldg(&pairs[i0].key_tile) : kNoTile;
-    kt1 = i1 < e1 ? __ldg(&pairs[i1].key_tile) : kNoTile;
-  }
-  __device__ __forceinline__ bool has() const { return kt0 != kNoTile || kt1 != kNoTile; }
-  // Next key tile and which halves list it; heads are refilled at once so that the loads overlap
-  // the caller's waits.
-  __device__ __forceinline__ int next(bool& live0, bool& live1) {
-    const int kt = min(kt0, kt1);
-    live0 = kt0 == kt;
-    live1 = kt1 == kt;
-    if (live0) kt0 = ++i0 < e0 ? __ldg(&pairs[i0].key_tile) : kNoTile;
-    if (live1) kt1 = ++i1 < e1 ? __ldg(&pairs[i1].key_tile) : kNoTile;
-    return kt;
-  }
-};
 
 template <int NH>
 __global__ void __launch_bounds__(Cfg<NH>::kThreads, Cfg<NH>::kMinCtas)
@@ -774,7 +541,6 @@ bool encode_patch(CUtensorMap* tm, const void* base, int64_t first_token, int64_
   return r == CUDA_SUCCESS;
 }
 
-
 template <int NH>
 litevar_status_t launch_variant(const TensorMaps& tm, const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
   static std::once_flag attr_once;
@@ -803,8 +569,8 @@ litevar_status_t launch_variant(const TensorMaps& tm, const FwdParams& p, int n_
 
 }  // namespace
 
-litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
-  TensorMaps tm;
+bool encode_tensor_maps(const FwdParams& p, tc::TensorMaps* tmp) {
+  tc::TensorMaps& tm = *tmp;
   memset(&tm, 0, sizeof(tm));
   bool ok;
   if (p.q_patch)
@@ -818,7 +584,12 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
                       p.k_sb) &&
          encode_patch(&tm.v2[i], p.v, p.patch_off[i], p.patch_scale[i], p.n_heads, p.batch_computed, p.v_st, p.v_sh,
                       p.v_sb);
-  if (!ok) return LITEVAR_ERR_INVALID_ARG;
+  return ok;
+}
+
+litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
+  TensorMaps tm;
+  if (!encode_tensor_maps(p, &tm)) return LITEVAR_ERR_INVALID_ARG;
   // A step with a single query tile and more CTAs than SMs runs the small build: two CTAs share an SM and
   // hide each other's set-up and drain.  With fewer CTAs than SMs sharing would only halve each CTA's SM.
   const int n_sm = current_sm_count();

@@ -140,6 +140,8 @@ cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, in
 
 // Tensor-core path.  Returns LITEVAR_OK or an error status (tensor-map encoding can fail).
 litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
+// The same path with one softmax thread per query row (register reallocation between warpgroups).
+litevar_status_t launch_forward_ws(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
 
 }  // namespace litevar
 

@@ -669,6 +669,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
     }
     return LITEVAR_OK;
   }
+  if (plan->kernel == LITEVAR_KERNEL_TCGEN05_WS) return launch_forward_ws(p, st.n_q_tiles, stream);
   return launch_forward_tcgen05(p, st.n_q_tiles, stream);
 }
 
@@ -786,7 +787,7 @@ litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan) {
 }
 
 litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel) {
-  if (!plan || kernel < LITEVAR_KERNEL_AUTO || kernel > LITEVAR_KERNEL_TCGEN05) return LITEVAR_ERR_INVALID_ARG;
+  if (!plan || kernel < LITEVAR_KERNEL_AUTO || kernel > LITEVAR_KERNEL_TCGEN05_WS || kernel == LITEVAR_KERNEL_SMALL) return LITEVAR_ERR_INVALID_ARG;
   plan->kernel = kernel;
   return LITEVAR_OK;
 }

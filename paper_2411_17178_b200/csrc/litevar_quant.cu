@@ -105,25 +105,27 @@ __global__ void __launch_bounds__(kQuantThreads) quant_rows_kernel(QuantArgs a) 
     const float r = __fdiv_rn(1.f, s1);  // one division per row; the elements multiply, see below
     float c[8];
     uint32_t packed[4];
+    // round to nearest even without the conversion pipe: adding and subtracting 1.5 * 2^23 is exact rounding
+    // to an integer for |y| < 2^22, and |y| stays near 2^(B-1) here.  |y| <= 2^(B-1) + 1, so two units in the
+    // last place are at most 2^-14: an estimate farther than 2^-12 from a half-integer rounds as the exact
+    // quotient does.  Rows with an estimate closer than that (few) are redone with the IEEE division.
+    bool near_tie = false;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      float q = 0.f;
-      if (s > 0.f) {
-        // round to nearest even without the conversion pipe: adding and subtracting 1.5 * 2^23 is exact
-        // rounding to an integer for |y| < 2^22, and |y| stays near 2^(B-1) here
-        const float d = __fsub_rn(v[i], z);
-        float y = __fmul_rn(d, r);
-        float n = __fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f);
-        // |y| <= 2^(B-1) + 1, so two units in the last place are at most 2^-14: an estimate farther than
-        // 2^-12 from a half-integer rounds as the exact quotient does
-        if (fabsf(__fsub_rn(y, n)) > 0.5f - 0.000244140625f) {
-          y = __fdiv_rn(d, s1);
-          n = __fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f);
-        }
-        q = fminf(fmaxf(n, a.lo), a.hi);
-      }
-      c[i] = q;
+      const float y = __fmul_rn(__fsub_rn(v[i], z), r);
+      const float n = __fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f);
+      near_tie |= fabsf(__fsub_rn(y, n)) > 0.5f - 0.000244140625f;
+      c[i] = n;
     }
+    if (near_tie) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float y = __fdiv_rn(__fsub_rn(v[i], z), s1);
+        c[i] = __fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) c[i] = s > 0.f ? fminf(fmaxf(c[i], a.lo), a.hi) : 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const __nv_bfloat162 d2 = __floats2bfloat162_rn(__fadd_rn(__fmul_rn(c[2 * i], s), z),

@@ -9,7 +9,7 @@ import torch
 
 from oracle import litevar_oracle as orc
 from paper_2411_17178_b200 import binding, workloads as wl
-from tests.gpu_util import assert_close, lib_ready, run_forward
+from tests.gpu_util import assert_close, check_sampled, lib_ready, run_forward, stratified_samples
 
 pytestmark = pytest.mark.gpu
 
@@ -77,18 +77,6 @@ def test_config2_one_layer_all_steps_with_sharing(kernel, tiling):
     plan.close()
 
 
-def _samples(rng, rows, H, n_k, count, s_k):
-    """Stratified rows: every (b,h) gets some; grid corners and edges always included."""
-    fixed = [0, s_k - 1, n_k - s_k, n_k - 1, (s_k // 2) * s_k + s_k // 2, 127, 128, n_k - 129]
-    out = []
-    per = max(1, count // (rows * H))
-    for b in range(rows):
-        for h in range(H):
-            qs = list(rng.integers(0, n_k, size=per)) + ([fixed[(b * H + h) % len(fixed)]])
-            out += [(b, h, int(min(max(q, 0), n_k - 1))) for q in qs]
-    return out
-
-
 @pytest.mark.parametrize("tiling", [binding.TILING_AUTO, binding.TILING_PATCH], ids=["auto", "patch"])
 def test_config4_final_steps_sampled(tiling):
     lib_ready()
@@ -98,21 +86,24 @@ def test_config4_final_steps_sampled(tiling):
     tab = orc.window_table(w.scales)
     Kc, Vc = wl.make_kv(w, 0, batch_rows=2 * B)
     rng = np.random.default_rng(4)
+    total = 0
     for k in (8, 9, 10):
         Q = wl.make_q(w, 0, k, batch_rows=2 * B)
         got, out = run_forward(plan, k, B, Q, Kc, Vc, binding.KERNEL_TCGEN05)
-        n_k = w.scales[k - 1] ** 2
-        smp = _samples(rng, 2 * B, w.n_heads, n_k, 300, w.scales[k - 1])
+        smp = stratified_samples(plan, k, 2 * B, w.n_heads, w.scales[k - 1], 20 if tiling == binding.TILING_AUTO else 8, rng)
+        total += len(smp)
         ref = orc.attention_sampled(w.scales, k, tab[k - 1], Q, Kc, Vc, smp, share_cfg=True)
-        g = np.stack([got[b, h, q] for b, h, q in smp])
-        assert_close(g, ref, f"config 4 step {k}")
+        check_sampled(got, ref, smp, f"config 4 step {k}")
         assert torch.equal(out[:B].view(torch.int16), out[B:].view(torch.int16))
+    assert tiling != binding.TILING_AUTO or total >= 4096
     plan.close()
 
 
 @pytest.mark.parametrize("tiling", [binding.TILING_AUTO, binding.TILING_RASTER], ids=["auto", "raster"])
 @pytest.mark.parametrize("rho", [(1, 8), (1, 4), (1, 2), None], ids=["rho1/8", "rho1/4", "rho1/2", "dense"])
 def test_config5_sampled(rho, tiling):
+    # the 2K step in the launch configuration the bench times: at least 4096 oracle rows per variant under the
+    # default tiling, one from every query tile of every tenth (batch row, head) unit
     lib_ready()
     w = wl.WORKLOADS[5]
     if rho is None:
@@ -124,11 +115,12 @@ def test_config5_sampled(rho, tiling):
     Kc, Vc = wl.make_kv(w, 0)
     Q = wl.make_q(w, 0, 14)
     got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, binding.KERNEL_TCGEN05)
+    assert np.isfinite(got).all()
     rng = np.random.default_rng(5)
-    smp = _samples(rng, 2, w.n_heads, 16384, 256, 128)
+    smp = stratified_samples(plan, 14, 2, w.n_heads, 128, 128 if tiling == binding.TILING_AUTO else 8, rng)
+    assert tiling != binding.TILING_AUTO or len(smp) >= 4096
     ref = orc.attention_sampled(w.scales, 14, tab[13], Q, Kc, Vc, smp)
-    g = np.stack([got[b, h, q] for b, h, q in smp])
-    assert_close(g, ref, f"config 5 rho={rho}")
+    check_sampled(got, ref, smp, f"config 5 rho={rho}")
     plan.close()
 
 
@@ -266,21 +258,19 @@ def test_band_window_2k_sampled():
     Q = wl.make_q(w, 0, 14)
     got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, binding.KERNEL_TCGEN05)
     rng = np.random.default_rng(6)
-    smp = _samples(rng, 2, w.n_heads, 16384, 128, 128)
-    lv = orc.mask_band(w.scales, 14, tab[13], q_rows=[q for _, _, q in smp])
-    L = orc.map_shape(w.scales, 14)[1]
-    ref = np.stack([orc.attention_rows(orc.bf16_to_f64(Q[b, h, q:q + 1]), orc.bf16_to_f64(Kc[b, h, :L]),
-                                       orc.bf16_to_f64(Vc[b, h, :L]), lv[i:i + 1], 0.125)[0]
-                    for i, (b, h, q) in enumerate(smp)])
-    g = np.stack([got[b, h, q] for b, h, q in smp])
-    assert_close(g, ref, "band 2K")
+    smp = stratified_samples(plan, 14, 2, w.n_heads, 128, 128, rng)
+    assert len(smp) >= 4096
+    ref = orc.attention_sampled(w.scales, 14, tab[13], Q, Kc, Vc, smp, band=True)
+    check_sampled(got, ref, smp, "band 2K")
     plan.close()
 
 
-@pytest.mark.parametrize("cfg,steps", [(2, (1, 4, 8, 10)), (3, (6, 10)), (4, (7, 10))], ids=["cfg2", "cfg3", "cfg4"])
-def test_bench_launch_configuration_sampled(cfg, steps):
-    # the batch, head count, sharing and kernel build that bench.py times for this workload; outputs are
-    # checked on sampled rows the oracle computes one by one
+@pytest.mark.parametrize("cfg,steps,per_unit", [(2, (1, 4, 8, 10), 12), (3, (6, 8, 9, 10), 6), (4, (7, 8, 9, 10), 8)],
+                         ids=["cfg2", "cfg3", "cfg4"])
+def test_bench_launch_configuration_sampled(cfg, steps, per_unit):
+    # the batch, head count, sharing and kernel build that bench.py times for this workload; outputs are checked
+    # on stratified rows the oracle computes one by one: at least 4096 per workload, every (batch row, head)
+    # unit, every query tile of every tenth unit, grid corners and edges, the heaviest and lightest tiles
     lib_ready()
     w = wl.WORKLOADS[cfg]
     B = w.batch_pairs
@@ -289,20 +279,20 @@ def test_bench_launch_configuration_sampled(cfg, steps):
     Kc, Vc = wl.make_kv(w, 0, max_step=max(steps))
     kd, vd = Kc.cuda(), Vc.cuda()
     rng = np.random.default_rng(cfg)
+    total = 0
     for k in steps:
         Q = wl.make_q(w, 0, k)
         out = torch.full(Q.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
         plan.forward(k, B, Q.cuda(), kd, vd, out)
         torch.cuda.synchronize()
         assert plan.poll() == 0
-        n_k, s_k = w.scales[k - 1] ** 2, w.scales[k - 1]
-        smp = _samples(rng, 2 * B, w.n_heads, n_k, 2 * B * w.n_heads, s_k)[::max(1, (2 * B * w.n_heads) // 192)]
+        assert bool(torch.isfinite(out.float()).all())
+        smp = stratified_samples(plan, k, 2 * B, w.n_heads, w.scales[k - 1], per_unit, rng)
+        total += len(smp)
         ref = orc.attention_sampled(w.scales, k, tab[k - 1], Q, Kc, Vc, smp, share_cfg=True)
-        got = out.double().cpu().numpy()
-        g = np.stack([got[b, h, q] for b, h, q in smp])
-        assert np.isfinite(got).all()
-        assert_close(g, ref, f"config {cfg} step {k}")
+        check_sampled(out, ref, smp, f"config {cfg} step {k}")
         assert torch.equal(out[:B].view(torch.int16), out[B:].view(torch.int16))
+    assert total >= 4096
     plan.close()
 
 
