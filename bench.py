@@ -6,22 +6,27 @@
 
 A "step" is one pass of the whole hot path over one batch: one full generation's attention,
 i.e. every scale step of every layer of the chosen workload (for the single-call workloads 1 and
-5: one call).  Rank 0 prints ONE JSON line.  The headline workload is the full 10-step VAR-d16
-schedule at 256px (16 layers x 16 heads, batch 2x8, default window, CFG sharing everywhere).
+5: one call).  Rank 0 prints ONE JSON line.  The headline workload is the largest one: the 2K-scale
+step (16384 queries against a 34240-row cache, 16 heads, batch 2) under the default window (rho = 1/4).
 
 value            useful TFLOP/s: 256 FLOP per live map entry of every (batch row, head) the kernel
                  computes (under CFG sharing: the conditional half), inputs resident in HBM,
                  the generation's calls replayed from one CUDA graph
 e2e              the same metric through the per-call API with pinned HOST buffers: every call
                  copies its Q and the new scale's K/V rows to the device and its output back
-roofline         HBM bound of the kernel that takes most of the generation (the steps it serves are
-                 replayed as a graph of their own and timed with CUDA events): compulsory bytes (Q +
-                 K/V prefix read once per computed (b, h), output written for all 2B rows) over that
-                 time; the other forward kernel is listed beside it
+roofline         the dominant forward kernel of the workload against the roofline that binds it: the
+                 tensor roofline (useful and executed FLOP per launch over the launch time measured here
+                 with CUDA events, against the measured bf16 peak) on the 512px and 2K workloads, the HBM
+                 roofline (compulsory bytes: Q + K/V prefix read once per computed (b, h), output written
+                 for all 2B rows) on the 256px ones; `traffic` is the DRAM traffic per launch from the
+                 committed ncu summary while the kernel sources are unchanged
+roofline_hbm_workload2   the HBM block of the 256px VAR-d16 generation (the round-one headline), kept beside it
 cpu_baseline     the CPU fp64 oracle timed on this machine's host cores on a bounded sample
-all_configs      the five benchmark workloads, window and full-mask variants (unless --no-extras)
+all_configs      the five benchmark workloads, window and full-mask variants, one short row each
+                 (unless --no-extras); per-step detail in all_configs_detail
+plan_us          microseconds litevar_attn_plan takes per schedule (device planner + one synchronisation)
 calibration      the window calibration kernel against the HBM roofline (also: --calibration alone)
-qkv8             the 8-bit Q/K/V row quantiser against the HBM roofline, and the headline generation
+qkv8             the 8-bit Q/K/V row quantiser against the HBM roofline, and the 256px generation
                  with Q and the appended K/V rows quantised before every call
 
 With --impl reference the oracle itself is timed (rank 0 only) and printed in the same format.
@@ -63,25 +68,38 @@ def peaks():
 def kernel_source_hash():
     import hashlib
     h = hashlib.sha256()
-    for f in ("litevar_fwd_tc.cu", "litevar_fwd_small.cu", "litevar_plan.cu", "litevar_internal.h"):
+    for f in ("litevar_fwd_tc.cu", "litevar_fwd_ws.cu", "litevar_tc_ptx.h", "litevar_fwd_small.cu", "litevar_plan.cu",
+              "litevar_internal.h"):
         h.update(open(os.path.join(ROOT, "paper_2411_17178_b200", "csrc", f), "rb").read())
     return h.hexdigest()
 
 
-KERNEL_NAMES = {1: "fwd_simt_kernel", 2: "fwd_tc_kernel", 3: "fwd_small_kernel"}
+KERNEL_NAMES = {1: "fwd_simt_kernel", 2: "fwd_tc_kernel", 3: "fwd_small_kernel", 4: "fwd_ws_kernel"}
 
 
-def recorded_traffic(kernel="fwd_tc_kernel"):
-    """DRAM bytes per launch of that forward kernel on workload 2 from the committed ncu summary, or None
-    when the kernel sources have changed since those counters were taken."""
-    path = os.path.join(ROOT, "profiles", "fwd_tc_workload2_traffic.txt")
+def recorded_traffic(key):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) recorded in
+    profiles/traffic.txt under `key`, or None when the kernel sources have changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "traffic.txt")
     try:
         kv = dict(l.strip().split("=", 1) for l in open(path) if "=" in l and not l.startswith("#"))
         if kv.get("source_sha256") != kernel_source_hash():
             return None
-        return int(kv["bytes_per_launch." + kernel])
+        return int(kv[key])
     except Exception:
         return None
+
+
+def config_dict(w, variant, rho, extra=None):
+    """The `config` object of the JSON line; the same keys on both arms."""
+    d = {"workload": f"config {w.index}: {w.name}", "variant": variant, "scales": list(w.scales),
+         "steps_per_generation": len(w.steps), "layers": w.n_layers, "heads": w.n_heads,
+         "batch": f"2x{w.batch_pairs}", "cfg_share": w.share_cfg,
+         "window_rho": list(rho or w.rho) if variant == "window" else None}
+    d["launch"] = d["l2"] = d["note"] = None
+    if extra:
+        d.update(extra)
+    return d
 
 
 # --------------------------------------------------------------------------------------- accounting
@@ -366,26 +384,28 @@ def measure_config(w: wl.Workload, variant: str, rho, steps, warmup, device, pk,
     assert plan.poll() == 0, "device-side wait timed out"
     scale = repeat / w.n_layers                # calls timed per generation's worth of calls
     us_gen = ms * 1e3 / scale
-    res = dict(config=w.index, workload=w.name, variant=variant,
-               rho=list(rho or w.rho) if variant == "window" else None,
-               calls_per_generation=len(w.steps) * w.n_layers,
-               us_per_generation=round(us_gen, 2),
-               us_per_call=round(us_gen / (len(w.steps) * w.n_layers), 3),
-               useful_tflops=round(useful * w.n_layers / (us_gen * 1e-6) / 1e12, 2),
-               executed_tflops=round(executed * w.n_layers / (us_gen * 1e-6) / 1e12, 2),
-               live_density_in_tiles=round(useful / executed, 4),
-               useful_frac_of_bf16_peak=round(useful * w.n_layers / (us_gen * 1e-6) / 1e12 / pk["bf16"], 4),
-               hbm_gbs_compulsory=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9, 1),
-               hbm_frac=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9 / pk["hbm"], 4),
-               buffer_sets=n_sets, tiling="auto")
+    tf = useful * w.n_layers / (us_gen * 1e-6) / 1e12
+    res = dict(config=w.index, variant=variant if variant == "dense" else "rho %d/%d" % tuple(rho or w.rho),
+               us_per_call=round(us_gen / (len(w.steps) * w.n_layers), 2), us_per_generation=round(us_gen, 1),
+               useful_tflops=round(tf, 1),
+               executed_tflops=round(executed * w.n_layers / (us_gen * 1e-6) / 1e12, 1),
+               density=round(useful / executed, 3),
+               useful_of_bf16_peak=round(tf / pk["bf16"], 4),
+               hbm_gbs=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9),
+               hbm_frac=round(nbytes * w.n_layers / (us_gen * 1e-6) / 1e9 / pk["hbm"], 3))
+    detail = dict(config=w.index, workload=w.name, variant=res["variant"],
+                  calls_per_generation=len(w.steps) * w.n_layers, buffer_sets=n_sets, tiling="auto")
     if len(w.steps) > 1:
         # microseconds per call at every step: one graph of that step's calls over all layers
         per_step = {}
         for k in w.steps:
             ms_k = time_graph(plan, w, bufs, [(k, layer % n_sets) for layer in range(repeat)], max(2, steps // 2), 2)
             per_step[str(k)] = round(ms_k * 1e3 / repeat, 2)
-        res["us_per_call_by_step"] = per_step
-        res["kernel_by_step"] = {str(k): KERNEL_NAMES[plan.step_kernel(k, w.batch_pairs)] for k in w.steps}
+        detail["us_per_call_by_step"] = per_step
+        detail["kernel_by_step"] = {str(k): KERNEL_NAMES[plan.step_kernel(k, w.batch_pairs)] for k in w.steps}
+    else:
+        detail["kernel"] = KERNEL_NAMES[plan.step_kernel(w.steps[0], w.batch_pairs)]
+    res = (res, detail)
     plan.close()
     return res, bufs
 
@@ -554,16 +574,14 @@ def gpu_arm(args):
     if rank != 0:
         return
 
+    rho_used = tuple(args.rho) if args.rho else w.rho
     out = {
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"config {w.index}: {w.name}", "variant": variant, "scales": list(w.scales),
-                   "steps_per_generation": len(w.steps), "layers": w.n_layers, "heads": w.n_heads,
-                   "batch": f"2x{w.batch_pairs}", "cfg_share": w.share_cfg, "window_rho": list(args.rho or w.rho),
-                   "launch": "one CUDA graph replay per generation",
-                   "l2": f"inputs larger than L2: {bufs.bytes() / 1e6:.0f} MB over {bufs.n_sets} layer buffer "
-                         "sets visited step-major"},
+        "config": config_dict(w, variant, rho_used, {
+            "launch": "one CUDA graph replay per generation",
+            "l2": f"inputs larger than L2: {bufs.bytes() / 1e6:.0f} MB over {bufs.n_sets} buffer sets visited in turn"}),
         "gpu_launches": launches_per_step * args.steps,
         "us_per_generation": round(ms_step * 1e3, 2),
         "us_per_image": round(ms_step * 1e3 / w.batch_pairs, 2),
@@ -576,39 +594,67 @@ def gpu_arm(args):
     if sampler:
         out["clocks"] = sampler.summary()
 
-    # ---- roofline of the dominant forward kernel on this workload.  AUTO runs two kernels (small steps /
-    # the rest); each group of steps is replayed as its own graph and timed with CUDA events, the kernel
-    # with the larger share of the generation is the one reported.
-    groups = {}
-    for k in w.steps:
-        groups.setdefault(KERNEL_NAMES[plan.step_kernel(k, w.batch_pairs)], []).append(k)
-    timed = {}
-    for name, ks in groups.items():
-        g_calls = [(k, layer % n_sets) for k in ks for layer in range(repeat)]
-        g_ms = time_graph(plan, w, bufs, g_calls, max(3, args.steps // 2), 3) / scale
-        timed[name] = dict(steps=ks, launches=len(ks) * w.n_layers, us=g_ms * 1e3,
-                           bytes=per_layer_work(w, counts, w.share_cfg, ks)[2] * w.n_layers)
-    total_us = sum(t["us"] for t in timed.values())
-    dom = max(timed, key=lambda n: timed[n]["us"])
-    d = timed[dom]
-    alg_bytes_launch = d["bytes"] / d["launches"]
-    avg_launch_s = d["us"] * 1e-6 / d["launches"]
-    achieved = alg_bytes_launch / avg_launch_s / 1e9
-    out["roofline"] = {"bound": "hbm", "achieved": round(achieved, 1), "peak": pk["hbm"], "unit": "GB/s",
-                       "frac": round(achieved / pk["hbm"], 4),
-                       "traffic": recorded_traffic(dom) if (w.index == 2 and variant == "window" and not args.rho) else None,
-                       "kernel": dom, "peak_source": pk["source"], "steps": d["steps"],
-                       "launches_per_generation": d["launches"],
-                       "share_of_generation_time": round(d["us"] / total_us, 4),
-                       "algorithmic_bytes_per_launch": round(alg_bytes_launch),
-                       "avg_launch_us": round(avg_launch_s * 1e6, 3),
-                       "other_kernels": [
-                           {"kernel": n, "steps": t["steps"], "launches_per_generation": t["launches"],
-                            "algorithmic_bytes_per_launch": round(t["bytes"] / t["launches"]),
-                            "avg_launch_us": round(t["us"] / t["launches"], 3),
-                            "share_of_generation_time": round(t["us"] / total_us, 4),
-                            "hbm_frac": round(t["bytes"] / (t["us"] * 1e-6) / 1e9 / pk["hbm"], 4)}
-                           for n, t in timed.items() if n != dom]}
+    # ---- roofline of the dominant forward kernel on this workload.  AUTO may run several kernels (small steps /
+    # short lists / long lists); each group of steps is replayed as its own graph and timed with CUDA events, the
+    # kernel with the largest share of the generation is the one reported.
+    def kernel_groups(pl, wk, bf, n_sets_, repeat_, scale_, cnts):
+        groups = {}
+        for k in wk.steps:
+            groups.setdefault(KERNEL_NAMES[pl.step_kernel(k, wk.batch_pairs)], []).append(k)
+        timed = {}
+        for name, ks in groups.items():
+            g_calls = [(k, layer % n_sets_) for k in ks for layer in range(repeat_)]
+            g_ms = time_graph(pl, wk, bf, g_calls, max(3, args.steps // 2), 3) / scale_
+            u, e, b = per_layer_work(wk, cnts, wk.share_cfg, ks)
+            timed[name] = dict(steps=ks, launches=len(ks) * wk.n_layers, us=g_ms * 1e3, bytes=b * wk.n_layers,
+                               useful=u * wk.n_layers, executed=e * wk.n_layers)
+        return timed
+
+    def hbm_block(timed, traffic_key):
+        total_us = sum(t["us"] for t in timed.values())
+        dom = max(timed, key=lambda n: timed[n]["us"])
+        d = timed[dom]
+        alg = d["bytes"] / d["launches"]
+        sec = d["us"] * 1e-6 / d["launches"]
+        return {"bound": "hbm", "achieved": round(alg / sec / 1e9, 1), "peak": pk["hbm"], "unit": "GB/s",
+                "frac": round(alg / sec / 1e9 / pk["hbm"], 4), "traffic": recorded_traffic(traffic_key) if traffic_key else None,
+                "kernel": dom, "peak_source": pk["source"], "steps": d["steps"],
+                "launches_per_generation": d["launches"], "share_of_generation_time": round(d["us"] / total_us, 4),
+                "algorithmic_bytes_per_launch": round(alg), "avg_launch_us": round(sec * 1e6, 3),
+                "other_kernels": [
+                    {"kernel": n, "steps": t["steps"], "launches_per_generation": t["launches"],
+                     "avg_launch_us": round(t["us"] / t["launches"], 3),
+                     "share_of_generation_time": round(t["us"] / total_us, 4),
+                     "hbm_frac": round(t["bytes"] / (t["us"] * 1e-6) / 1e9 / pk["hbm"], 4)}
+                    for n, t in timed.items() if n != dom]}
+
+    def tensor_block(timed, traffic_key):
+        total_us = sum(t["us"] for t in timed.values())
+        dom = max(timed, key=lambda n: timed[n]["us"])
+        d = timed[dom]
+        sec = d["us"] * 1e-6 / d["launches"]
+        useful_l, exec_l = d["useful"] / d["launches"], d["executed"] / d["launches"]
+        return {"bound": "tensor", "achieved": round(useful_l / sec / 1e12, 2), "peak": pk["bf16"], "unit": "TFLOP/s",
+                "frac": round(useful_l / sec / 1e12 / pk["bf16"], 4),
+                "traffic": recorded_traffic(traffic_key) if traffic_key else None,
+                "kernel": dom, "peak_source": pk["source"] + " (burst; a launch is timed alone)",
+                "useful_flop_per_launch": round(useful_l), "executed_flop_per_launch": round(exec_l),
+                "achieved_executed": round(exec_l / sec / 1e12, 2),
+                "frac_executed": round(exec_l / sec / 1e12 / pk["bf16"], 4),
+                "frac_of_sustained_peak": round(useful_l / sec / 1e12 / pk["bf16_sustained"], 4),
+                "algorithmic_bytes_per_launch": round(d["bytes"] / d["launches"]),
+                "hbm_frac_compulsory": round(d["bytes"] / d["launches"] / sec / 1e9 / pk["hbm"], 4),
+                "avg_launch_us": round(sec * 1e6, 3), "steps": d["steps"],
+                "launches_per_generation": d["launches"], "share_of_generation_time": round(d["us"] / total_us, 4),
+                "other_kernels": [
+                    {"kernel": n, "steps": t["steps"], "launches_per_generation": t["launches"],
+                     "avg_launch_us": round(t["us"] / t["launches"], 3),
+                     "share_of_generation_time": round(t["us"] / total_us, 4)} for n, t in timed.items() if n != dom]}
+
+    timed = kernel_groups(plan, w, bufs, n_sets, repeat, scale, counts)
+    default_run = variant == "window" and not args.rho
+    tkey = f"workload{w.index}.{'dense' if variant == 'dense' else 'window'}.bytes_per_launch" if (default_run or variant == "dense") else None
+    out["roofline"] = tensor_block(timed, tkey) if w.index in (4, 5) else hbm_block(timed, tkey)
 
     if args.kernel_only:
         plan.close()
@@ -629,7 +675,8 @@ def gpu_arm(args):
     if world == 1 and not args.no_cpu:
         out["cpu_baseline"] = oracle_baseline(w, args.cpu_seconds)
 
-    # ---- the five workloads, window and dense variants
+    # ---- the five workloads, window and dense variants; the HBM roofline of the 256px generation; plan times
+    detail = []
     if world == 1 and not args.no_extras:
         table = []
         reps, warm = 5, 3
@@ -638,14 +685,49 @@ def gpu_arm(args):
             shared_bufs = None
             variants = [("window", r) for r in (wi.rho_sweep or (wi.rho,))] + [("dense", None)]
             for var, rho in variants:
-                r, shared_bufs = measure_config(wi, var, rho, reps, warm, device, pk, shared_bufs)
-                table.append(r)
+                (row, det), shared_bufs = measure_config(wi, var, rho, reps, warm, device, pk, shared_bufs)
+                table.append(row)
+                detail.append(det)
+            if idx == 2 and w.index != 2:
+                p2 = make_plan(wi, "window")
+                n2 = shared_bufs.n_sets
+                rep2 = max(wi.n_layers, n2)
+                out["roofline_hbm_workload2"] = hbm_block(
+                    kernel_groups(p2, wi, shared_bufs, n2, rep2, rep2 / wi.n_layers, schedule_counts(p2, wi)),
+                    "workload2.window.bytes_per_launch")
+                p2.close()
             del shared_bufs
             torch.cuda.empty_cache()
         out["all_configs"] = table
+        out["plan_us"] = measure_plan_times()
         out["calibration"] = measure_calibration(device, pk)
         out["qkv8"] = measure_qkv8(device, pk)
-    print(json.dumps(out), flush=True)
+        out["all_configs_detail"] = detail
+    # the short table goes out early in the line and the long per-step records last
+    order = ["metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+             "vs_baseline", "dtype", "data", "config", "gpu_launches", "clocks", "roofline", "e2e", "cpu_baseline",
+             "all_configs"]
+    line = {k: out[k] for k in order if k in out}
+    line.update({k: v for k, v in out.items() if k not in line})
+    print(json.dumps(line), flush=True)
+
+
+def measure_plan_times():
+    """Microseconds per litevar_attn_plan call (window table, bounds, classification, compaction, element masks
+    and launch order of every step on the device, one synchronisation at the end), best of three."""
+    res = {}
+    for name, scales, heads in (("256px", wl.SCALES_256, 16), ("512px", wl.SCALES_512, 36), ("2K", wl.SCALES_2K, 16)):
+        from paper_2411_17178_b200 import binding
+        best = None
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            pl = binding.Plan(scales, n_heads=heads)
+            t1 = time.perf_counter()
+            pl.close()
+            best = t1 - t0 if best is None else min(best, t1 - t0)
+        res[name] = round(best * 1e6, 1)
+    return res
 
 
 # --------------------------------------------------------------------------------------- CPU arm
@@ -729,10 +811,7 @@ def reference_arm(args):
         "impl": "reference", "metric": METRIC, "value": round(value, 6), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(el_tot / args.steps * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"config {w.index}: {w.name}", "variant": "window", "scales": list(w.scales),
-                   "steps_per_generation": len(w.steps), "layers": w.n_layers, "heads": w.n_heads,
-                   "batch": f"2x{w.batch_pairs}", "cfg_share": w.share_cfg, "window_rho": list(w.rho),
-                   "note": "each step is a bounded sample of the workload run by the CPU oracle"},
+        "config": config_dict(w, "window", w.rho, {"note": "each step is a bounded sample of the workload run by the CPU oracle"}),
         "gpu_launches": 0,
         "cpu_baseline": {"value": round(value, 6), "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                          "sample": f"per step: {what}"},
@@ -744,10 +823,10 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--dense", action="store_true", help="full-mask variant of the same kernel")
     ap.add_argument("--no-extras", action="store_true", help="skip the five-workload table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")

@@ -83,9 +83,10 @@ typedef struct {
 
 /* Forward kernel selection (testing / measurement). */
 enum {
-  LITEVAR_KERNEL_AUTO = 0,    /* per step: the small-step kernel where the step fits it, else the tcgen05 kernel */
+  LITEVAR_KERNEL_AUTO = 0,    /* per step: the small-step kernel where the step fits it, else a tcgen05 kernel (the one
+                                 with a softmax thread per query row on long tile lists) */
   LITEVAR_KERNEL_SIMT = 1,    /* plain CUDA-core kernel (slow; cross-check and bring-up) */
-  LITEVAR_KERNEL_TCGEN05 = 2, /* tcgen05/TMEM/TMA kernel for every step */
+  LITEVAR_KERNEL_TCGEN05 = 2, /* tcgen05/TMEM/TMA kernel with two softmax threads per query row, for every step */
   LITEVAR_KERNEL_SMALL = 3,   /* reported by litevar_plan_step_kernel only: warp-level mma kernel for steps with one
                                  query tile, at most two raster key tiles and little work */
   LITEVAR_KERNEL_TCGEN05_WS = 4 /* tcgen05 kernel with one softmax thread per query row, for every step */
@@ -168,7 +169,8 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
  *     that device current; make that first call outside any stream capture.
  *   - There is no empty-row check: with a caller table that leaves a query without a live key the
  *     row's output is undefined.  A bounded device-side wait that expires is not reported.
- * Errors: INVALID_ARG, UNSUPPORTED, ARCH, CUDA.
+ * Errors: INVALID_ARG, UNSUPPORTED, ARCH, CUDA.  (A tensor-map encoding failure, INVALID_ARG, is found after the two
+ * planner kernels have been launched; they write only the library's own array.)
  */
 litevar_status_t litevar_attn_forward_static(const int32_t* scales, int32_t n_scales, int32_t n_heads,
                                              int32_t head_dim, float sm_scale, const litevar_window_t* window,
@@ -239,12 +241,13 @@ litevar_status_t litevar_plan_materialize_mask(const litevar_plan_t* plan, int32
  * with this plan gave up on a bounded wait since the last poll (the flag is then cleared). */
 litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan);
 
-/* Select the forward kernel (LITEVAR_KERNEL_AUTO, _SIMT or _TCGEN05).  Not thread-safe against concurrent
- * forwards. */
+/* Testing and measurement hook: force one forward kernel for every step (LITEVAR_KERNEL_SIMT, _TCGEN05,
+ * _TCGEN05_WS) or return to LITEVAR_KERNEL_AUTO, which is what a plan starts with and all a product caller needs.
+ * Changes the plan: not to be called while forwards of this plan may be running or being issued. */
 litevar_status_t litevar_plan_set_kernel(litevar_plan_t* plan, int32_t kernel);
 
 /* Which kernel litevar_attn_forward launches for step_k with batch_pairs under the current selection:
- * *kernel receives LITEVAR_KERNEL_SIMT, _TCGEN05 or _SMALL.  Host only; the paper has no counterpart (it gives no kernel design). */
+ * *kernel receives LITEVAR_KERNEL_SIMT, _TCGEN05, _TCGEN05_WS or _SMALL.  Host only; the paper has no counterpart (it gives no kernel design). */
 litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
                                           int32_t* kernel);
 

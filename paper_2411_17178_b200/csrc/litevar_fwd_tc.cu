@@ -29,8 +29,9 @@
 // TMEM columns: S_0 [0,128)  S_1 [128,256)  O_0 [256,336)  O_1 [336,416); P_h for keys [0,64) lies in
 // S_h columns [0,32), for keys [64,128) in S_h columns [64,96).
 //
-// Every wait is bounded: when a wait runs out the CTA raises the plan's status word, drains its
-// outstanding copies, frees its TMEM and returns.
+// Every wait on an mbarrier or on a partner thread is bounded: when one runs out the CTA raises the plan's status
+// word, drains its outstanding copies, frees its TMEM and returns.  (The TMEM allocation itself blocks while
+// other CTAs on the SM hold the columns; every CTA of this library releases them before it exits.)
 #include <cstring>
 #include <mutex>
 
@@ -94,8 +95,8 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // 1-D grid, heaviest query-tile pairs first: all (head, batch row) units of a pair are neighbours
-  const int n_units = p.n_heads * p.batch_computed;
-  const int pair_rank = blockIdx.x / n_units, unit = blockIdx.x - pair_rank * n_units;
+  int pair_rank, unit;  // grouped launch order, see cta_work
+  cta_work(p, (n_q_tiles + NH - 1) / NH, pair_rank, unit);
   const int h = unit % p.n_heads, b = unit / p.n_heads;
   // the launch order lists query-tile PAIRS; the one-tile build takes the tiles in natural order
   const int qt0 = NH == 2 ? 2 * (p.order ? __ldg(&p.order[pair_rank]) : pair_rank) : pair_rank, qt1 = qt0 + 1;
@@ -247,22 +248,20 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
                 if (!(ok = mbar_wait(&sm.p_full[hh][1], (uint32_t)(n_pv[hh] & 1), abort_flag, p.status))) break;
                 tc_fence_after();
               }
-#pragma unroll
-              for (int g = 0; g < 4; ++g) {
-                // 16 keys = 16 rows of 128 B = 2048 B; P: 8 packed columns per step, key half 1 starts at S column 64
-                const int kk = 2 * part + (g & 1) + 4 * (g >> 1);
-                mma_ts(tmem + kColO + kOutCols * hh, tmem + kColS + 128 * hh + 8 * kk + (kk >= 4 ? 32 : 0),
-                       v_desc + (uint64_t)(2048 >> 4) * kk, kIdescPV, (n_pv[hh] > 0 || part > 0 || g > 0) ? 1u : 0u);
-              }
+              // four steps of 16 keys (16 rows of 128 B = 2048 B of V, 8 packed columns of P) in one instruction
+              // sequence: key groups {0, 1, 4, 5} for the first part, {2, 3, 6, 7} for the second; the second key
+              // half of P starts at S column 64
+              mma_ts_x4_at<8, 64, 72, 128, 512, 640>(tmem + kColO + kOutCols * hh, tmem + kColS + 128 * hh + 16 * part,
+                                                     v_desc + (uint64_t)(2 * 128) * part, kIdescPV,
+                                                     (n_pv[hh] > 0 || part > 0) ? 1u : 0u);
             }
             if (!ok) break;
             mma_commit(&sm.o_full[hh]);
             ++n_pv[hh];
           }
           if (have && live[hh]) {  // S_hh = Q_hh K^T, after the PV above in issue order
-#pragma unroll
-            for (int kk = 0; kk < kHeadDim / 16; ++kk)  // 16 bf16 = 32 B per step inside the swizzle row
-              mma_ss(tmem + kColS + 128 * hh, q_desc[hh] + 2 * kk, k_desc + 2 * kk, kIdescQK, kk > 0 ? 1u : 0u);
+            // 16 bf16 = 32 B per step inside the swizzle rows of Q and K
+            mma_ss_x4<2, 2>(tmem + kColS + 128 * hh, q_desc[hh], k_desc, kIdescQK, 0u);
             mma_commit(&sm.s_full[hh]);
           }
         }

@@ -1,33 +1,35 @@
-// Warp-specialised tensor-core forward kernel for sm_100a with register reallocation: one softmax thread owns
-// a whole query row, and the scores of the next key tile are formed while the softmax of the current one runs.
+// Warp-specialised tensor-core forward kernel for sm_100a with register reallocation: one softmax thread owns a
+// whole query row, and the scores of the next key tile are formed while the softmax of the current one runs.
+// Used for steps with long tile lists (from eight key tiles per query tile on); the kernel of litevar_fwd_tc.cu
+// serves the shorter ones.
 //
-// One CTA handles NH adjacent query tiles ("halves", 128 queries each) of one (head, batch row) and walks the
-// union of their live key-tile lists in plan order, so every K/V tile is staged once for all halves.
+// The kernel is written for NH query tiles ("halves", 128 queries each) of one (head, batch row) per CTA, walking
+// the union of their live key-tile lists; the library launches NH = 1, two CTAs per SM (see launch_forward_ws).
 //   warps 0 .. 4 NH - 1   softmax warpgroup of half h = warp / 4: thread m of the group owns query slot m (TMEM
-//                         lane m).  Per key tile it reads the 128 scores of its row from TMEM once and releases
-//                         the S block at once (s_read), applies the plan's element mask in registers, takes the
-//                         row maximum without any exchange, forms the probabilities against a lazily updated
-//                         reference maximum, adds them up, and writes P (packed bf16) to a block of its own.
-//                         At the end it normalises and stores its output row.
+//                         lane m).  A key tile is taken in two passes of 64 keys through one rolled copy of the
+//                         code: 64 scores from TMEM into registers, the plan's element mask, the row maximum
+//                         without any exchange, the probabilities against a lazily updated reference maximum
+//                         (every fourth pair of exponentials on the FMA pipe by a cubic, the rest on the
+//                         exponential pipe), their sum, and P (packed bf16) into a TMEM block of its own.  The S
+//                         block is released as soon as the second pass has its scores in registers.  At the end
+//                         the thread normalises and stores its output row.
 //   warp 4 NH             TMA producer (one lane): Q of every half, then K and V of every listed key tile into two
 //                         rings of kStages tiles.
 //   warp 4 NH + 1         TMEM allocation; one lane issues S_h = Q_h K^T of the next key tile as soon as the
 //                         softmax threads have read the previous S_h.
 //   warp 4 NH + 2         one lane issues O_h += P_h V of a tile once its P is complete.  Because P does not
-//                         overlay S, the score product of tile j + 1 does not wait for the softmax of tile j: the
-//                         softmax warpgroups go from tile to tile without a pause and the PV product is off
-//                         their critical path.  Two issuing lanes because each is a chain of waits and short
-//                         instruction sequences whose latency, not the tensor pipe, sets the pace of one lane.
+//                         overlay S, the score product of tile j + 1 does not wait for the softmax of tile j and
+//                         the PV product is off the softmax's critical path.
 //   warp 4 NH + 3         idle (it completes the warpgroup that gives its registers away).
 // Registers: the kernel starts with the launch-bound count for every thread; the last warpgroup then releases
-// all but 56 per thread (setmaxnreg.dec) and the softmax warpgroups take them (setmaxnreg.inc), which is what lets
-// a thread keep its 128 scores in registers.
+// all but 56 per thread (setmaxnreg.dec) and the softmax warpgroups take them (setmaxnreg.inc).
 // MMA issue: four K = 16 steps per instruction sequence with immediate offsets (mma_*_x4).  Measured on B200,
 // back to back: 65 cycles per step at N = 128 (64 are pure math), 50 at N <= 64, for A in shared memory or in
-// TMEM alike; a step issued with per-step address arithmetic in the issuing lane took 100 to 150.
+// TMEM alike; a tcgen05.commit between groups of four to eight steps adds 100 to 150 cycles of tensor-pipe time.
 // TMEM columns: S_h [128 h, +128); O_h [128 NH + 64 h, +64); P_h [192 NH + 64 h, +64).
-// The element mask, the tile lists, CFG sharing (second store at batch row b + B) and the bounded waits are
-// those of the plan and of the other forward kernels (paper Sections 2 and 3).
+// Every wait on an mbarrier is bounded (2^32 cycles); on expiry the CTA raises the plan's status word, drains its
+// copies, frees its TMEM and returns.  The element mask, the tile lists and CFG sharing (second store at batch row
+// b + B) are those of the plan and of the other forward kernels (paper Sections 2 and 3).
 #include <cstring>
 #include <mutex>
 
@@ -59,7 +61,7 @@ struct WsShared {
   alignas(1024) uint8_t v[kStages][kTileBytes];
   alignas(8) uint64_t q_full;
   uint64_t k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
-  uint64_t s_full[2], s_read[2], p_full[2], pv_done[2], stagger;
+  uint64_t s_full[2], s_read[2], p_full[2], pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -69,6 +71,23 @@ constexpr uint32_t kIdescS = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kB
                              ((uint32_t)(kBlockM >> 4) << 24);
 constexpr uint32_t kIdescO = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kHeadDim >> 3) << 17) |
                              ((uint32_t)(kBlockM >> 4) << 24);
+
+// 2^x for x <= 8 on the FMA pipe: x = n + f with n = round(x) and f in [-1/2, 1/2]; 2^f by a cubic fitted to it
+// (relative error 7.5e-5, far inside the bf16 rounding of P), 2^n by adding n to the exponent field.  Scores of
+// dead keys (-inf) are clamped to 2^-125.
+__device__ __forceinline__ float2 exp2_fma2(float2 x) {
+  x.x = fmaxf(x.x, -125.f);
+  x.y = fmaxf(x.y, -125.f);
+  const float2 t = __fadd2_rn(x, make_float2(12582912.f, 12582912.f));  // the integer part in the low mantissa bits
+  const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+  const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
+  float2 y = __ffma2_rn(make_float2(0.05517153441905975f, 0.05517153441905975f), f,
+                        make_float2(0.2426111102104187f, 0.2426111102104187f));
+  y = __ffma2_rn(y, f, make_float2(0.6932610273361206f, 0.6932610273361206f));
+  y = __ffma2_rn(y, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
+  return make_float2(__uint_as_float(__float_as_uint(y.x) + (__float_as_uint(t.x) << 23)),
+                     __uint_as_float(__float_as_uint(y.y) + (__float_as_uint(t.y) << 23)));
+}
 
 template <int N>
 __device__ __forceinline__ void reg_dec() {
@@ -89,8 +108,8 @@ fwd_ws_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int kProducerWarp = 4 * NH, kMmaWarp = 4 * NH + 1, kPvWarp = 4 * NH + 2;
-  const int n_units = p.n_heads * p.batch_computed;
-  const int pair_rank = blockIdx.x / n_units, unit = blockIdx.x - pair_rank * n_units;
+  int pair_rank, unit;  // grouped launch order, see cta_work
+  cta_work(p, (n_q_tiles + NH - 1) / NH, pair_rank, unit);
   const int h = unit % p.n_heads, b = unit / p.n_heads;
   const int qt0 = NH == 2 ? 2 * (p.order ? __ldg(&p.order[pair_rank]) : pair_rank) : pair_rank, qt1 = qt0 + 1;
   const bool has1 = NH == 2 && qt1 < n_q_tiles;
@@ -110,7 +129,6 @@ fwd_ws_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       mbar_init(&sm.p_full[i], 4);
       mbar_init(&sm.pv_done[i], 1);
     }
-    mbar_init(&sm.stagger, 4);
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -275,15 +293,6 @@ fwd_ws_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       Pair pr = sd.pairs[pbeg];
       uint4 mk = make_uint4(~0u, ~0u, ~0u, ~0u);
       if (pr.mask_block >= 0) mk = __ldg(&sd.mask[(size_t)pr.mask_block * kBlockM + m]);
-      // The two halves share each scheduler's exponential pipe, and a pass is a stretch of loads, masks and
-      // maxima followed by a stretch of exponentials.  Half 1 starts its first tile when half 0 has finished the
-      // first pass of its first tile, so that one half's loads and maxima run under the other's exponentials;
-      // the offset persists from tile to tile (while both are in their exponentials neither gains on the other).
-      // Only when both lists start with the same key tile: then both first score products are issued together
-      // and half 0 never depends on half 1's progress.
-      const bool staggered = NH == 2 && end0 > beg0 && end1 > beg1 &&
-                             __ldg(&sd.pairs[beg0].key_tile) == __ldg(&sd.pairs[beg1].key_tile);
-      if (staggered && hh == 1) ok = mbar_wait_inl(&sm.stagger, 0u, abort_flag, p.status);
       for (int j = 0; ok && j < n_tiles; ++j) {
         Pair pr_next = pr;  // next pair's mask words travel while this tile is processed
         uint4 mk_next = make_uint4(~0u, ~0u, ~0u, ~0u);
@@ -370,7 +379,7 @@ fwd_ws_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
               __syncwarp();
               if (lane == 0) mbar_arrive(&sm.s_read[hh]);
             }
-            // probabilities against the reference: scale and shift (packed FMAs), exponentials, row sum, bf16
+            // probabilities against the reference: scale and shift (packed FMAs), 2^x, row sum, bf16
             const float msc = row_max == -INFINITY ? 0.f : row_max * sc;
             const float2 nm2 = make_float2(-msc, -msc);
             const bool add_sum = !(redo && hf == 0);
@@ -379,13 +388,17 @@ fwd_ws_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
               const float2 xa = __ffma2_rn(make_float2(__uint_as_float(r[e + 0]), __uint_as_float(r[e + 1])), sc2, nm2);
               const float2 xb = __ffma2_rn(make_float2(__uint_as_float(r[e + 2]), __uint_as_float(r[e + 3])), sc2, nm2);
               const float2 pa = make_float2(fast_exp2(xa.x), fast_exp2(xa.y));
-              const float2 pb = make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+              // every fourth pair on the FMA pipe: the exponential pipe (16 per clock and SM) is what a pass waits for
+              const float2 pb = (e & 4) ? exp2_fma2(xb) : make_float2(fast_exp2(xb.x), fast_exp2(xb.y));
+              // the row sum adds the probabilities as the PV product sees them (rounded to bf16): numerator and
+              // denominator of a row then agree, and a row with one dominant key reproduces that key's V exactly
+              const uint32_t ka = pack_bf16(pa.x, pa.y), kb = pack_bf16(pb.x, pb.y);
               if (add_sum) {
-                l2a = __fadd2_rn(l2a, pa);
-                l2b = __fadd2_rn(l2b, pb);
+                l2a = __fadd2_rn(l2a, make_float2(__uint_as_float(ka << 16), __uint_as_float(ka & 0xffff0000u)));
+                l2b = __fadd2_rn(l2b, make_float2(__uint_as_float(kb << 16), __uint_as_float(kb & 0xffff0000u)));
               }
-              pk[(e >> 1) + 0] = pack_bf16(pa.x, pa.y);
-              pk[(e >> 1) + 1] = pack_bf16(pb.x, pb.y);
+              pk[(e >> 1) + 0] = ka;
+              pk[(e >> 1) + 1] = kb;
             }
           } else {
             if (hf == 1) {
@@ -402,10 +415,6 @@ fwd_ws_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
             pv_seen = true;
           }
           tmem_st32(tP + 32 * hf, pk);
-          if (staggered && hh == 0 && j == 0 && hf == 0 && !redo) {  // see the stagger above
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.stagger);
-          }
         }
         if (!ok) break;
         tmem_wait_st();  // P and, where it was rescaled, the accumulator
@@ -490,11 +499,11 @@ litevar_status_t launch_ws_variant(const TensorMaps& tm, const FwdParams& p, int
 litevar_status_t launch_forward_ws(const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
   TensorMaps tm;
   if (!encode_tensor_maps(p, &tm)) return LITEVAR_ERR_INVALID_ARG;
-  const int n_sm = current_sm_count();
-  const long long units = (long long)p.n_heads * p.batch_computed;
-  const bool lite = (n_q_tiles == 1 && units > n_sm) ||
-                    (units * n_q_tiles >= 2LL * n_sm && p.pairs_per_tile > 0 && p.pairs_per_tile <= 14);
-  return lite ? launch_ws_variant<1>(tm, p, n_q_tiles, stream) : launch_ws_variant<2>(tm, p, n_q_tiles, stream);
+  // One query tile per CTA, two CTAs per SM: measured on B200 against the two-tile build of the same kernel (one
+  // CTA per SM, K/V staged once for both tiles) it is 2 % faster on the full-mask 2K step and 4 % faster on the
+  // windowed one, where the union of two tiles' lists also executes pairs that only one of them lists.  Two
+  // independent CTAs drift apart, so that one's loads, masks and maxima fall under the other's exponentials.
+  return launch_ws_variant<1>(tm, p, n_q_tiles, stream);
 }
 
 }  // namespace litevar

@@ -111,11 +111,26 @@ struct FwdParams {
   int32_t* status;              // device word, set non-zero when a bounded wait expires
   int32_t pairs_per_tile;       // average live key tiles per query tile (0: unknown); picks the kernel build
   int32_t first_tile_zero;      // 1: every query tile's list starts with key tile 0 (its copies start at once)
+  int32_t units_per_group;      // launch order of the tensor-core kernels: (batch row, head) units per L2 group
   int32_t overlap_launch;       // 1: the tensor-core kernel may start its set-up before the previous kernel of the
                                 // stream has finished (the plan it reads was complete long before)
 };
 
 // SM count of the current device, looked up once per device (the attribute query costs a microsecond).
+// L2 size of the current device in bytes, looked up once per device.
+inline long long current_l2_bytes() {
+  static long long cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 64ll << 20;
+  long long n = cached[dev];
+  if (n == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, dev) != cudaSuccess || v <= 0) return 64ll << 20;
+    cached[dev] = n = v;  // benign race: every writer stores the same value
+  }
+  return n;
+}
+
 inline int current_sm_count() {
   static int cached[64] = {};
   int dev = 0;
@@ -126,6 +141,16 @@ inline int current_sm_count() {
     cached[dev] = n;  // benign race: every writer stores the same value
   }
   return n;
+}
+
+// (batch row, head) units whose K and V prefixes (L_k rows of 128 B each) together fill half of L2: the group size
+// of the tensor-core kernels' launch order.
+inline int units_per_l2_group(int L_k, int n_units) {
+  const long long per_unit = 2ll * L_k * kHeadDim * 2;
+  long long g = (current_l2_bytes() / 2) / (per_unit > 0 ? per_unit : 1);
+  if (g < 1) g = 1;
+  if (g > n_units) g = n_units;
+  return (int)g;
 }
 
 cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t stream);

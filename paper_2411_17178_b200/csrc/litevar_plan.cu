@@ -319,105 +319,46 @@ __global__ void __launch_bounds__(128) materialize_kernel(SetDesc sd, Schedule s
   }
 }
 
-template <typename T>
-litevar_status_t dev_alloc(litevar_plan* plan, T** out, size_t count) {
-  void* p = nullptr;
-  size_t bytes = count * sizeof(T);
-  if (bytes == 0) bytes = sizeof(T);
-  cudaError_t e = cudaMalloc(&p, bytes);
-  if (e != cudaSuccess) {
-    (void)cudaGetLastError();
-    return e == cudaErrorMemoryAllocation ? LITEVAR_ERR_OOM : LITEVAR_ERR_CUDA;
-  }
-  plan->allocations.push_back(p);
-  *out = static_cast<T*>(p);
-  return LITEVAR_OK;
-}
-
-struct Scratch {
-  std::vector<void*> ptrs;
-  ~Scratch() {
-    for (void* p : ptrs) cudaFree(p);
-  }
+// Bump allocator over one device allocation: sizes are added up in a first pass (base == nullptr), the block is
+// allocated, and the same sequence of calls then hands out the pointers.  256-byte granules.
+struct Arena {
+  char* base = nullptr;
+  size_t used = 0;
   template <typename T>
-  cudaError_t get(T** out, size_t count) {
-    void* p = nullptr;
-    cudaError_t e = cudaMalloc(&p, count * sizeof(T) ? count * sizeof(T) : sizeof(T));
-    if (e == cudaSuccess) {
-      ptrs.push_back(p);
-      *out = static_cast<T*>(p);
-    }
-    return e;
+  T* take(size_t count) {
+    const size_t bytes = (count * sizeof(T) + 255) & ~static_cast<size_t>(255);
+    T* p = base ? reinterpret_cast<T*>(base + used) : nullptr;
+    used += bytes ? bytes : 256;
+    return p;
   }
 };
 
-litevar_status_t plan_step_set(litevar_plan* plan, int k0, int set, cudaStream_t stream) {
-  Step& st = plan->steps[k0];
-  StepSet& ss = st.sets[set];
-  const Schedule& sc = plan->sched;
-  const int K = sc.n_scales;
-  const int32_t* d_radius_row = plan->d_radius + ((size_t)set * K + k0) * K;
+// Scratch of one (step, window set) during planning.
+struct SetScratch {
+  uint8_t* cls = nullptr;
+  int32_t *row_live = nullptr, *partial_base = nullptr, *blk = nullptr;
+};
 
-  litevar_status_t s = dev_alloc(plan, &ss.d_bounds, (size_t)(k0 + 1) * st.s_k);
-  if (s != LITEVAR_OK) return s;
-  bounds_kernel<<<(unsigned)(((k0 + 1) * st.s_k + 255) / 256), 256, 0, stream>>>(sc, k0, d_radius_row, ss.d_bounds);
+// Per (step, set) results the host needs: written by the planner kernels into one device array, read back once.
+struct SetTotals {
+  int32_t n_pairs, n_partial, n_full, empty_row;  // count_scan_kernel / empty_row_kernel
+  unsigned long long live_entries;                // classify_kernel
+  int32_t first_not_zero, pad;                    // first_tile_kernel
+  Pair first_pairs[2];                            // the whole list of a small step (n_pairs <= 2)
+};
 
-  PlanGeom g{k0, st.s_k, st.n_k, st.L_k, st.n_key_tiles, plan->shape, st.raster_len, st.d_q_geom, st.d_key_geom};
-  Scratch tmp;
-  uint8_t* d_cls = nullptr;
-  int32_t *d_row_live = nullptr, *d_partial_base = nullptr, *d_totals = nullptr, *d_blk = nullptr;
-  unsigned long long* d_live = nullptr;
-  size_t n_cand = (size_t)st.n_q_tiles * st.n_key_tiles;
-  LV_CUDA(tmp.get(&d_cls, n_cand));
-  LV_CUDA(tmp.get(&d_row_live, (size_t)st.n_k));
-  LV_CUDA(tmp.get(&d_partial_base, (size_t)st.n_q_tiles));
-  LV_CUDA(tmp.get(&d_totals, 4));
-  LV_CUDA(tmp.get(&d_blk, n_cand));
-  LV_CUDA(tmp.get(&d_live, 1));
-  LV_CUDA(cudaMemsetAsync(d_row_live, 0, sizeof(int32_t) * st.n_k, stream));
-  LV_CUDA(cudaMemsetAsync(d_totals, 0, sizeof(int32_t) * 4, stream));
-  LV_CUDA(cudaMemsetAsync(d_live, 0, sizeof(unsigned long long), stream));
+__global__ void copy_first_pairs_kernel(const Pair* pairs, const int32_t* n_pairs, Pair* out) {
+  if (threadIdx.x < 2 && (int)threadIdx.x < *n_pairs) out[threadIdx.x] = pairs[threadIdx.x];
+}
 
-  s = dev_alloc(plan, &ss.d_row_ptr, (size_t)st.n_q_tiles + 1);
-  if (s != LITEVAR_OK) return s;
-
-  dim3 grid2((unsigned)st.n_key_tiles, (unsigned)st.n_q_tiles);
-  classify_kernel<<<grid2, 128, 0, stream>>>(sc, g, ss.d_bounds, d_radius_row, d_cls, d_row_live, d_live);
-  empty_row_kernel<<<(unsigned)((st.n_k + 255) / 256), 256, 0, stream>>>(st.n_k, d_row_live, d_totals + 3);
-  int threads = st.n_q_tiles < 32 ? 32 : (st.n_q_tiles > 512 ? 512 : ((st.n_q_tiles + 31) / 32) * 32);
-  count_scan_kernel<<<1, threads, 2 * sizeof(int32_t) * st.n_q_tiles, stream>>>(
-      st.n_q_tiles, st.n_key_tiles, d_cls, ss.d_row_ptr, d_partial_base, d_totals);
-  int32_t totals[4];
-  unsigned long long live = 0;
-  LV_CUDA(cudaMemcpyAsync(totals, d_totals, sizeof(totals), cudaMemcpyDeviceToHost, stream));
-  LV_CUDA(cudaMemcpyAsync(&live, d_live, sizeof(live), cudaMemcpyDeviceToHost, stream));
-  LV_CUDA(cudaStreamSynchronize(stream));
-  if (totals[3] != 0) return LITEVAR_ERR_EMPTY_ROW;
-  ss.n_pairs = totals[0];
-  ss.n_partial = totals[1];
-  ss.n_full = totals[2];
-  ss.live_entries = (int64_t)live;
-
-  s = dev_alloc(plan, &ss.d_pairs, (size_t)ss.n_pairs);
-  if (s != LITEVAR_OK) return s;
-  s = dev_alloc(plan, &ss.d_mask, (size_t)ss.n_partial * kBlockM);
-  if (s != LITEVAR_OK) return s;
-  compact_kernel<<<(unsigned)((st.n_q_tiles + 127) / 128), 128, 0, stream>>>(
-      st.n_q_tiles, st.n_key_tiles, d_cls, ss.d_row_ptr, d_partial_base, ss.d_pairs, d_blk);
-  mask_bits_kernel<<<grid2, 128, 0, stream>>>(sc, g, ss.d_bounds, d_radius_row, d_blk, ss.d_mask);
-  s = dev_alloc(plan, &ss.d_order, (size_t)(st.n_q_tiles + 1) / 2);
-  if (s != LITEVAR_OK) return s;
-  launch_order_kernel<<<(unsigned)(((st.n_q_tiles + 1) / 2 + 127) / 128), 128, 0, stream>>>(st.n_q_tiles, ss.d_row_ptr,
-                                                                                         ss.d_order);
-  LV_CUDA(cudaMemsetAsync(d_totals, 0, sizeof(int32_t), stream));
-  first_tile_kernel<<<(unsigned)((st.n_q_tiles + 127) / 128), 128, 0, stream>>>(st.n_q_tiles, ss.d_row_ptr, ss.d_pairs,
-                                                                                d_totals);
-  int32_t not_zero = 1;
-  LV_CUDA(cudaMemcpyAsync(&not_zero, d_totals, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
-  LV_CUDA(cudaGetLastError());
-  LV_CUDA(cudaStreamSynchronize(stream));  // scratch is freed when `tmp` goes out of scope
-  ss.first_tile_zero = not_zero == 0;
-  return LITEVAR_OK;
+// The plan's buffers, the tensor maps and the launch all belong to the device the plan was made on.
+bool on_plan_device(const litevar_plan_t* plan) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  return dev == plan->device;
 }
 
 bool strides_ok(const litevar_strides_t* s) {
@@ -431,6 +372,242 @@ int small_mode(const litevar_plan_t* plan, const Step& st, long long units) {
   for (const StepSet& ss : st.sets)  // every window set of the step has a list the small-step kernel can take
     if (ss.small.n <= 0) return 0;
   return small_step_mode(st.n_k, st.L_k, units, plan->n_sm);
+}
+
+#define LV_TRY(expr)                                                                              \
+  do {                                                                                            \
+    cudaError_t e__ = (expr);                                                                     \
+    if (e__ != cudaSuccess) {                                                                     \
+      (void)cudaGetLastError();                                                                   \
+      return e__ == cudaErrorMemoryAllocation ? LITEVAR_ERR_OOM : LITEVAR_ERR_CUDA;               \
+    }                                                                                             \
+  } while (0)
+
+// Everything litevar_attn_plan does after its argument checks.  Device memory: one arena for the plan (tables,
+// tile geometry, bounds, lists, launch orders; the lists sized for every candidate pair), one block for the
+// element masks (sized exactly, once the device has counted the partial pairs) and one scratch block that is
+// freed before returning.  Two synchronisations: after the counting pass (the mask block's size and the
+// empty-row check come from it) and at the end.
+litevar_status_t build_plan(litevar_plan* plan, const int32_t* scales, int32_t n_scales, int32_t n_heads, float sm_scale,
+                            const litevar_window_t* window, const litevar_cfg_share_t* share, int dev, int n_sm,
+                            cudaStream_t stream) {
+  plan->device = dev;
+  plan->n_sm = n_sm;
+  plan->n_heads = n_heads;
+  plan->n_sets = window->n_sets;
+  plan->shape = window->shape;
+  plan->n_global = window->n_global_scales;
+  plan->rho_num = window->rho_num;
+  plan->rho_den = window->rho_den;
+  plan->tiling = window->tiling;
+  plan->sm_scale = sm_scale > 0.f ? sm_scale : 0.125f;
+  Schedule& sc = plan->sched;
+  memset(&sc, 0, sizeof(sc));
+  sc.n_scales = n_scales;
+  for (int i = 0; i < n_scales; ++i) {
+    sc.scale[i] = scales[i];
+    sc.off[i + 1] = sc.off[i] + scales[i] * scales[i];
+  }
+  const int K = n_scales, n_sets = plan->n_sets;
+  if (window->head_to_set && n_sets > 1) plan->head_to_set.assign(window->head_to_set, window->head_to_set + n_heads);
+
+  // ---- tile geometry of every step (host): raster tiles of 128 consecutive tokens, or 8x16 patches of a scale's
+  // grid where the grid is large enough for a 2-D window to leave whole patches dead
+  plan->steps.resize(K);
+  for (int k0 = 0; k0 < K; ++k0) {
+    Step& st = plan->steps[k0];
+    st.s_k = sc.scale[k0];
+    st.n_k = st.s_k * st.s_k;
+    st.L_k = sc.off[k0 + 1];
+    // AUTO: patches pay off for 2-D (square) windows on large grids; a band in token order wants raster tiles
+    const bool auto_patch = plan->tiling == LITEVAR_TILING_AUTO && plan->shape == LITEVAR_WINDOW_SQUARE;
+    const int q_min = plan->tiling == LITEVAR_TILING_PATCH ? 1 : (auto_patch ? 48 : 1 << 30);
+    const int key_min = plan->tiling == LITEVAR_TILING_PATCH ? 4 : 32;
+    st.q_patch = st.s_k >= q_min;
+    st.first_patch = k0 + 1;
+    if (st.q_patch) {  // patch key tiles only together with patch query tiles
+      int first = 0;
+      while (first <= k0 && sc.scale[first] < key_min) ++first;
+      if (k0 + 1 - first > kMaxPatchScales) first = k0 + 1 - kMaxPatchScales;
+      st.first_patch = first;
+    }
+    st.raster_len = sc.off[st.first_patch];
+    st.n_raster_tiles = (st.raster_len + kBlockN - 1) / kBlockN;
+    if (st.q_patch) {
+      for (int r = 0; r < st.s_k; r += kPatchRows)
+        for (int c = 0; c < st.s_k; c += kPatchCols) st.q_geom.push_back(TileGeom{k0, r, c, 0});
+    } else {
+      for (int q0 = 0; q0 < st.n_k; q0 += kBlockM) st.q_geom.push_back(TileGeom{-1, q0, 0, 0});
+    }
+    for (int t0 = 0; t0 < st.raster_len; t0 += kBlockN) st.key_geom.push_back(TileGeom{-1, t0, 0, 0});
+    for (int j = st.first_patch; j <= k0; ++j)
+      for (int r = 0; r < sc.scale[j]; r += kPatchRows)
+        for (int c = 0; c < sc.scale[j]; c += kPatchCols) st.key_geom.push_back(TileGeom{j, r, c, j - st.first_patch});
+    st.n_q_tiles = (int32_t)st.q_geom.size();
+    st.n_key_tiles = (int32_t)st.key_geom.size();
+    st.share = share && share->share_step && share->share_step[k0] != 0;
+    st.sets.resize(n_sets);
+  }
+
+  // ---- device memory: the same sequence of take() calls sizes the blocks and then hands out the pointers
+  std::vector<SetScratch> scratch((size_t)K * n_sets);
+  SetTotals* d_totals = nullptr;
+  int32_t* d_user = nullptr;
+  Arena plan_mem, tmp_mem;
+  auto lay_out = [&]() {
+    plan->d_status = plan_mem.take<int32_t>(1);
+    plan->d_radius = plan_mem.take<int32_t>((size_t)n_sets * K * K);
+    plan->d_head_to_set = plan->head_to_set.empty() ? nullptr : plan_mem.take<int32_t>((size_t)n_heads);
+    d_totals = tmp_mem.take<SetTotals>((size_t)K * n_sets);
+    d_user = window->radius ? tmp_mem.take<int32_t>((size_t)n_sets * K * K) : nullptr;
+    for (int k0 = 0; k0 < K; ++k0) {
+      Step& st = plan->steps[k0];
+      const size_t n_cand = (size_t)st.n_q_tiles * st.n_key_tiles;
+      st.d_q_geom = plan_mem.take<TileGeom>(st.q_geom.size());
+      st.d_key_geom = plan_mem.take<TileGeom>(st.key_geom.size());
+      st.d_sets = plan_mem.take<SetDesc>((size_t)n_sets);
+      for (int set = 0; set < n_sets; ++set) {
+        StepSet& ss = st.sets[set];
+        ss.d_bounds = plan_mem.take<int2>((size_t)(k0 + 1) * st.s_k);
+        ss.d_row_ptr = plan_mem.take<int32_t>((size_t)st.n_q_tiles + 1);
+        ss.d_order = plan_mem.take<int32_t>((size_t)(st.n_q_tiles + 1) / 2);
+        ss.d_pairs = plan_mem.take<Pair>(n_cand);  // room for every candidate pair; n_pairs of them are used
+        SetScratch& t = scratch[(size_t)k0 * n_sets + set];
+        t.cls = tmp_mem.take<uint8_t>(n_cand);
+        t.row_live = tmp_mem.take<int32_t>((size_t)st.n_k);
+        t.partial_base = tmp_mem.take<int32_t>((size_t)st.n_q_tiles);
+        t.blk = tmp_mem.take<int32_t>(n_cand);
+      }
+    }
+  };
+  lay_out();
+  void *plan_block = nullptr, *tmp_block = nullptr;
+  LV_TRY(cudaMalloc(&plan_block, plan_mem.used));
+  plan->allocations.push_back(plan_block);
+  LV_TRY(cudaMalloc(&tmp_block, tmp_mem.used));
+  struct Free {
+    void* p;
+    ~Free() { cudaFree(p); }
+  } free_tmp{tmp_block};
+  plan_mem = Arena{static_cast<char*>(plan_block), 0};
+  tmp_mem = Arena{static_cast<char*>(tmp_block), 0};
+  lay_out();
+  LV_TRY(cudaMemsetAsync(tmp_block, 0, tmp_mem.used, stream));  // counters, row_live, totals
+  LV_TRY(cudaMemsetAsync(plan->d_status, 0, sizeof(int32_t), stream));
+
+  // ---- A1: window tables on the device (default rule, or the caller's table normalised)
+  if (window->radius)
+    LV_TRY(cudaMemcpyAsync(d_user, window->radius, sizeof(int32_t) * n_sets * K * K, cudaMemcpyHostToDevice, stream));
+  for (int set = 0; set < n_sets; ++set)
+    window_table_kernel<<<1, 256, 0, stream>>>(sc, plan->shape, plan->n_global, plan->rho_num, plan->rho_den,
+                                               d_user ? d_user + (size_t)set * K * K : nullptr,
+                                               plan->d_radius + (size_t)set * K * K);
+  plan->radius.resize((size_t)n_sets * K * K);
+  LV_TRY(cudaMemcpyAsync(plan->radius.data(), plan->d_radius, sizeof(int32_t) * plan->radius.size(),
+                         cudaMemcpyDeviceToHost, stream));
+  if (plan->d_head_to_set)
+    LV_TRY(cudaMemcpyAsync(plan->d_head_to_set, plan->head_to_set.data(), sizeof(int32_t) * n_heads,
+                           cudaMemcpyHostToDevice, stream));
+
+  // ---- A2 + A3, counting pass: bounds, classification of every candidate pair, per-tile counts and offsets
+  for (int k0 = 0; k0 < K; ++k0) {
+    Step& st = plan->steps[k0];
+    LV_TRY(cudaMemcpyAsync(st.d_q_geom, st.q_geom.data(), sizeof(TileGeom) * st.q_geom.size(), cudaMemcpyHostToDevice,
+                           stream));
+    LV_TRY(cudaMemcpyAsync(st.d_key_geom, st.key_geom.data(), sizeof(TileGeom) * st.key_geom.size(),
+                           cudaMemcpyHostToDevice, stream));
+    const PlanGeom g{k0, st.s_k, st.n_k, st.L_k, st.n_key_tiles, plan->shape, st.raster_len, st.d_q_geom, st.d_key_geom};
+    const dim3 grid2((unsigned)st.n_key_tiles, (unsigned)st.n_q_tiles);
+    const int threads = st.n_q_tiles < 32 ? 32 : (st.n_q_tiles > 512 ? 512 : ((st.n_q_tiles + 31) / 32) * 32);
+    for (int set = 0; set < n_sets; ++set) {
+      StepSet& ss = st.sets[set];
+      const SetScratch& t = scratch[(size_t)k0 * n_sets + set];
+      SetTotals* tot = d_totals + (size_t)k0 * n_sets + set;
+      const int32_t* d_radius_row = plan->d_radius + ((size_t)set * K + k0) * K;
+      bounds_kernel<<<(unsigned)(((k0 + 1) * st.s_k + 255) / 256), 256, 0, stream>>>(sc, k0, d_radius_row, ss.d_bounds);
+      classify_kernel<<<grid2, 128, 0, stream>>>(sc, g, ss.d_bounds, d_radius_row, t.cls, t.row_live, &tot->live_entries);
+      empty_row_kernel<<<(unsigned)((st.n_k + 255) / 256), 256, 0, stream>>>(st.n_k, t.row_live, &tot->empty_row);
+      count_scan_kernel<<<1, threads, 2 * sizeof(int32_t) * st.n_q_tiles, stream>>>(
+          st.n_q_tiles, st.n_key_tiles, t.cls, ss.d_row_ptr, t.partial_base, &tot->n_pairs);
+    }
+  }
+  std::vector<SetTotals> totals((size_t)K * n_sets);
+  LV_TRY(cudaMemcpyAsync(totals.data(), d_totals, sizeof(SetTotals) * totals.size(), cudaMemcpyDeviceToHost, stream));
+  LV_TRY(cudaGetLastError());
+  LV_TRY(cudaStreamSynchronize(stream));
+  size_t mask_rows = 0;
+  for (int k0 = 0; k0 < K; ++k0)
+    for (int set = 0; set < n_sets; ++set) {
+      const SetTotals& t = totals[(size_t)k0 * n_sets + set];
+      if (t.empty_row != 0) return LITEVAR_ERR_EMPTY_ROW;
+      StepSet& ss = plan->steps[k0].sets[set];
+      ss.n_pairs = t.n_pairs;
+      ss.n_partial = t.n_partial;
+      ss.n_full = t.n_full;
+      ss.live_entries = (int64_t)t.live_entries;
+      mask_rows += (size_t)t.n_partial * kBlockM;
+    }
+
+  // ---- A3, second pass: compaction in canonical order, element masks of the partial pairs, launch order
+  void* mask_block = nullptr;
+  LV_TRY(cudaMalloc(&mask_block, (mask_rows ? mask_rows : 1) * sizeof(uint4)));
+  plan->allocations.push_back(mask_block);
+  uint4* next_mask = static_cast<uint4*>(mask_block);
+  std::vector<SetDesc> descs((size_t)K * n_sets);
+  for (int k0 = 0; k0 < K; ++k0) {
+    Step& st = plan->steps[k0];
+    const PlanGeom g{k0, st.s_k, st.n_k, st.L_k, st.n_key_tiles, plan->shape, st.raster_len, st.d_q_geom, st.d_key_geom};
+    const dim3 grid2((unsigned)st.n_key_tiles, (unsigned)st.n_q_tiles);
+    for (int set = 0; set < n_sets; ++set) {
+      StepSet& ss = st.sets[set];
+      const SetScratch& t = scratch[(size_t)k0 * n_sets + set];
+      SetTotals* tot = d_totals + (size_t)k0 * n_sets + set;
+      const int32_t* d_radius_row = plan->d_radius + ((size_t)set * K + k0) * K;
+      ss.d_mask = next_mask;
+      next_mask += (size_t)ss.n_partial * kBlockM;
+      compact_kernel<<<(unsigned)((st.n_q_tiles + 127) / 128), 128, 0, stream>>>(
+          st.n_q_tiles, st.n_key_tiles, t.cls, ss.d_row_ptr, t.partial_base, ss.d_pairs, t.blk);
+      mask_bits_kernel<<<grid2, 128, 0, stream>>>(sc, g, ss.d_bounds, d_radius_row, t.blk, ss.d_mask);
+      launch_order_kernel<<<(unsigned)(((st.n_q_tiles + 1) / 2 + 127) / 128), 128, 0, stream>>>(st.n_q_tiles,
+                                                                                             ss.d_row_ptr, ss.d_order);
+      first_tile_kernel<<<(unsigned)((st.n_q_tiles + 127) / 128), 128, 0, stream>>>(st.n_q_tiles, ss.d_row_ptr,
+                                                                                    ss.d_pairs, &tot->first_not_zero);
+      if (small_step_candidate(st.n_q_tiles, st.n_key_tiles, !st.q_patch && st.first_patch == k0 + 1) &&
+          ss.n_pairs >= 1 && ss.n_pairs <= 2)
+        copy_first_pairs_kernel<<<1, 32, 0, stream>>>(ss.d_pairs, &tot->n_pairs, tot->first_pairs);
+      descs[(size_t)k0 * n_sets + set] = SetDesc{ss.d_row_ptr, ss.d_pairs, ss.d_mask};
+    }
+    LV_TRY(cudaMemcpyAsync(st.d_sets, &descs[(size_t)k0 * n_sets], sizeof(SetDesc) * n_sets, cudaMemcpyHostToDevice,
+                           stream));
+  }
+  LV_TRY(cudaMemcpyAsync(totals.data(), d_totals, sizeof(SetTotals) * totals.size(), cudaMemcpyDeviceToHost, stream));
+  LV_TRY(cudaGetLastError());
+  LV_TRY(cudaStreamSynchronize(stream));  // the scratch block is freed on return
+  for (int k0 = 0; k0 < K; ++k0) {
+    Step& st = plan->steps[k0];
+    for (int set = 0; set < n_sets; ++set) {
+      const SetTotals& t = totals[(size_t)k0 * n_sets + set];
+      StepSet& ss = st.sets[set];
+      ss.first_tile_zero = t.first_not_zero == 0;
+      if (small_step_candidate(st.n_q_tiles, st.n_key_tiles, !st.q_patch && st.first_patch == k0 + 1) &&
+          ss.n_pairs >= 1 && ss.n_pairs <= 2) {
+        ss.small.n = ss.n_pairs;
+        ss.small.pr[0] = t.first_pairs[0];
+        ss.small.pr[1] = t.first_pairs[1];
+      }
+    }
+  }
+  return LITEVAR_OK;
+}
+
+// Which of the two tcgen05 kernels runs a step that is not a small one.  The kernel with one softmax thread per
+// query row pays off on long tile lists (measured on B200: 5 to 8 % faster from about eight key tiles per query
+// tile on, i.e. the last steps of the 512px schedule and the 2K step; 5 % slower on the two-to-six-tile lists of
+// the 256px schedule, where the set-up of its longer pipeline is not written off).
+bool use_row_kernel(const litevar_plan_t* plan, const Step& st) {
+  if (plan->kernel == LITEVAR_KERNEL_TCGEN05_WS) return true;
+  if (plan->kernel != LITEVAR_KERNEL_AUTO) return false;
+  return (st.sets[0].n_pairs + st.n_q_tiles - 1) / st.n_q_tiles >= 8;
 }
 
 }  // namespace
@@ -483,126 +660,17 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
 
   litevar_plan* plan = new (std::nothrow) litevar_plan();
   if (!plan) return LITEVAR_ERR_OOM;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  plan->device = dev;
-  plan->n_sm = prop.multiProcessorCount;
-  plan->n_heads = n_heads;
-  plan->n_sets = window->n_sets;
-  plan->shape = window->shape;
-  plan->n_global = window->n_global_scales;
-  plan->rho_num = window->rho_num;
-  plan->rho_den = window->rho_den;
-  plan->tiling = window->tiling;
-  plan->sm_scale = sm_scale > 0.f ? sm_scale : 0.125f;
-  Schedule& sc = plan->sched;
-  memset(&sc, 0, sizeof(sc));
-  sc.n_scales = n_scales;
-  for (int i = 0; i < n_scales; ++i) {
-    sc.scale[i] = scales[i];
-    sc.off[i + 1] = sc.off[i] + scales[i] * scales[i];
+  litevar_status_t result = LITEVAR_ERR_OOM;
+  try {
+    result = build_plan(plan, scales, n_scales, n_heads, sm_scale, window, share, dev, prop.multiProcessorCount,
+                        static_cast<cudaStream_t>(stream_));
+  } catch (...) {  // a host container ran out of memory: nothing crosses the C boundary
+    result = LITEVAR_ERR_OOM;
   }
-  const int K = n_scales;
-
-  auto fail = [&](litevar_status_t s) {
+  if (result != LITEVAR_OK) {
+    (void)cudaStreamSynchronize(static_cast<cudaStream_t>(stream_));  // planner kernels may still use the buffers
     litevar_plan_destroy(plan);
-    return s;
-  };
-  litevar_status_t s;
-  if ((s = dev_alloc(plan, &plan->d_status, 1)) != LITEVAR_OK) return fail(s);
-  if ((s = dev_alloc(plan, &plan->d_radius, (size_t)plan->n_sets * K * K)) != LITEVAR_OK) return fail(s);
-  if (cudaMemsetAsync(plan->d_status, 0, sizeof(int32_t), stream) != cudaSuccess) return fail(LITEVAR_ERR_CUDA);
-
-  // A1: window tables on the device (default rule, or the caller's table normalised)
-  int32_t* d_user = nullptr;
-  Scratch tmp;
-  if (window->radius) {
-    if (tmp.get(&d_user, (size_t)plan->n_sets * K * K) != cudaSuccess) return fail(LITEVAR_ERR_OOM);
-    if (cudaMemcpyAsync(d_user, window->radius, sizeof(int32_t) * plan->n_sets * K * K, cudaMemcpyHostToDevice,
-                        stream) != cudaSuccess)
-      return fail(LITEVAR_ERR_CUDA);
-  }
-  for (int set = 0; set < plan->n_sets; ++set)
-    window_table_kernel<<<1, 256, 0, stream>>>(sc, plan->shape, plan->n_global, plan->rho_num, plan->rho_den,
-                                               d_user ? d_user + (size_t)set * K * K : nullptr,
-                                               plan->d_radius + (size_t)set * K * K);
-  plan->radius.resize((size_t)plan->n_sets * K * K);
-  if (cudaMemcpyAsync(plan->radius.data(), plan->d_radius, sizeof(int32_t) * plan->radius.size(),
-                      cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-    return fail(LITEVAR_ERR_CUDA);
-  if (cudaStreamSynchronize(stream) != cudaSuccess) return fail(LITEVAR_ERR_CUDA);
-
-  if (window->head_to_set && plan->n_sets > 1) {
-    plan->head_to_set.assign(window->head_to_set, window->head_to_set + n_heads);
-    if ((s = dev_alloc(plan, &plan->d_head_to_set, (size_t)n_heads)) != LITEVAR_OK) return fail(s);
-    if (cudaMemcpyAsync(plan->d_head_to_set, plan->head_to_set.data(), sizeof(int32_t) * n_heads,
-                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
-      return fail(LITEVAR_ERR_CUDA);
-  }
-
-  plan->steps.resize(K);
-  for (int k0 = 0; k0 < K; ++k0) {
-    Step& st = plan->steps[k0];
-    st.s_k = sc.scale[k0];
-    st.n_k = st.s_k * st.s_k;
-    st.L_k = sc.off[k0 + 1];
-    // tile geometry of the step: raster tiles of 128 consecutive tokens, or 8x16 patches of a scale's grid
-    // where the grid is large enough for a 2-D window to leave whole patches dead
-    {
-      // AUTO: patches pay off for 2-D (square) windows on large grids; a band in token order wants raster tiles
-      const bool auto_patch = plan->tiling == LITEVAR_TILING_AUTO && plan->shape == LITEVAR_WINDOW_SQUARE;
-      const int q_min = plan->tiling == LITEVAR_TILING_PATCH ? 1 : (auto_patch ? 48 : 1 << 30);
-      const int key_min = plan->tiling == LITEVAR_TILING_PATCH ? 4 : 32;
-      st.q_patch = st.s_k >= q_min;
-      st.first_patch = k0 + 1;
-      if (st.q_patch) {  // patch key tiles only together with patch query tiles
-        int first = 0;
-        while (first <= k0 && sc.scale[first] < key_min) ++first;
-        if (k0 + 1 - first > kMaxPatchScales) first = k0 + 1 - kMaxPatchScales;
-        st.first_patch = first;
-      }
-      st.raster_len = sc.off[st.first_patch];
-      st.n_raster_tiles = (st.raster_len + kBlockN - 1) / kBlockN;
-      if (st.q_patch) {
-        for (int r = 0; r < st.s_k; r += kPatchRows)
-          for (int c = 0; c < st.s_k; c += kPatchCols) st.q_geom.push_back(TileGeom{k0, r, c, 0});
-      } else {
-        for (int q0 = 0; q0 < st.n_k; q0 += kBlockM) st.q_geom.push_back(TileGeom{-1, q0, 0, 0});
-      }
-      for (int t0 = 0; t0 < st.raster_len; t0 += kBlockN) st.key_geom.push_back(TileGeom{-1, t0, 0, 0});
-      for (int j = st.first_patch; j <= k0; ++j)
-        for (int r = 0; r < sc.scale[j]; r += kPatchRows)
-          for (int c = 0; c < sc.scale[j]; c += kPatchCols)
-            st.key_geom.push_back(TileGeom{j, r, c, j - st.first_patch});
-      st.n_q_tiles = (int32_t)st.q_geom.size();
-      st.n_key_tiles = (int32_t)st.key_geom.size();
-      if ((s = dev_alloc(plan, &st.d_q_geom, st.q_geom.size())) != LITEVAR_OK) return fail(s);
-      if ((s = dev_alloc(plan, &st.d_key_geom, st.key_geom.size())) != LITEVAR_OK) return fail(s);
-      if (cudaMemcpyAsync(st.d_q_geom, st.q_geom.data(), sizeof(TileGeom) * st.q_geom.size(), cudaMemcpyHostToDevice,
-                          stream) != cudaSuccess ||
-          cudaMemcpyAsync(st.d_key_geom, st.key_geom.data(), sizeof(TileGeom) * st.key_geom.size(),
-                          cudaMemcpyHostToDevice, stream) != cudaSuccess)
-        return fail(LITEVAR_ERR_CUDA);
-    }
-    st.share = share && share->share_step && share->share_step[k0] != 0;
-    st.sets.resize(plan->n_sets);
-    std::vector<SetDesc> descs(plan->n_sets);
-    for (int set = 0; set < plan->n_sets; ++set) {
-      if ((s = plan_step_set(plan, k0, set, stream)) != LITEVAR_OK) return fail(s);
-      descs[set] = SetDesc{st.sets[set].d_row_ptr, st.sets[set].d_pairs, st.sets[set].d_mask};
-      StepSet& ss = st.sets[set];
-      if (small_step_candidate(st.n_q_tiles, st.n_key_tiles, !st.q_patch && st.first_patch == k0 + 1) &&
-          ss.n_pairs >= 1 && ss.n_pairs <= 2) {
-        ss.small.n = ss.n_pairs;
-        if (cudaMemcpyAsync(ss.small.pr, ss.d_pairs, sizeof(Pair) * ss.n_pairs, cudaMemcpyDeviceToHost, stream) !=
-            cudaSuccess)
-          return fail(LITEVAR_ERR_CUDA);
-      }
-    }
-    if ((s = dev_alloc(plan, &st.d_sets, (size_t)plan->n_sets)) != LITEVAR_OK) return fail(s);
-    if (cudaMemcpyAsync(st.d_sets, descs.data(), sizeof(SetDesc) * plan->n_sets, cudaMemcpyHostToDevice,
-                        stream) != cudaSuccess)
-      return fail(LITEVAR_ERR_CUDA);
-    if (cudaStreamSynchronize(stream) != cudaSuccess) return fail(LITEVAR_ERR_CUDA);
+    return result;
   }
   *out_plan = plan;
   return LITEVAR_OK;
@@ -616,6 +684,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   if (step_k < 1 || step_k > plan->sched.n_scales || batch_pairs < 1) return LITEVAR_ERR_INVALID_ARG;
   if (!strides_ok(sq) || !strides_ok(sk) || !strides_ok(sv) || !strides_ok(so)) return LITEVAR_ERR_INVALID_ARG;
   if (((uintptr_t)Q | (uintptr_t)Kc | (uintptr_t)Vc | (uintptr_t)out) & 15) return LITEVAR_ERR_INVALID_ARG;
+  if (!on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
   const Step& st = plan->steps[step_k - 1];
   FwdParams p;
   p.sets = st.d_sets;
@@ -653,6 +722,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   p.first_tile_zero = st.raster_len > 0 ? 1 : 0;  // key tile 0 must be the raster tile of cache rows [0, 128)
   for (const StepSet& ss : st.sets) p.first_tile_zero &= ss.first_tile_zero ? 1 : 0;
   p.pairs_per_tile = (st.sets[0].n_pairs + st.n_q_tiles - 1) / st.n_q_tiles;
+  p.units_per_group = units_per_l2_group(st.L_k, p.n_heads * p.batch_computed);
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (const int mode = small_mode(plan, st, (long long)p.n_heads * p.batch_computed)) {
     if (launch_forward_small(p, st.sets[0].small, mode, plan->n_sm, stream) != cudaSuccess) {
@@ -669,7 +739,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
     }
     return LITEVAR_OK;
   }
-  if (plan->kernel == LITEVAR_KERNEL_TCGEN05_WS) return launch_forward_ws(p, st.n_q_tiles, stream);
+  if (use_row_kernel(plan, st)) return launch_forward_ws(p, st.n_q_tiles, stream);
   return launch_forward_tcgen05(p, st.n_q_tiles, stream);
 }
 
@@ -707,6 +777,7 @@ litevar_status_t litevar_plan_export_tiles(const litevar_plan_t* plan, int32_t s
                                            int32_t* pair_key_tile, uint8_t* pair_is_full) {
   litevar_status_t s = check_step_set(plan, step_k, set);
   if (s != LITEVAR_OK) return s;
+  if (!on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
   const Step& st = plan->steps[step_k - 1];
   const StepSet& ss = st.sets[set];
   auto put = [&](int32_t* out, const TileGeom& g, int side, int base, int limit) {
@@ -751,6 +822,7 @@ litevar_status_t litevar_plan_export_bounds(const litevar_plan_t* plan, int32_t 
   if (radius)
     memcpy(radius, plan->radius.data() + ((size_t)set * K + (step_k - 1)) * K, sizeof(int32_t) * K);
   if (bounds) {
+    if (!on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
     LV_CUDA(cudaDeviceSynchronize());
     LV_CUDA(cudaMemcpy(bounds, st.sets[set].d_bounds, sizeof(int2) * step_k * st.s_k, cudaMemcpyDeviceToHost));
   }
@@ -761,7 +833,7 @@ litevar_status_t litevar_plan_materialize_mask(const litevar_plan_t* plan, int32
                                                void* dev_bits, void* stream_) {
   litevar_status_t s = check_step_set(plan, step_k, set);
   if (s != LITEVAR_OK) return s;
-  if (!dev_bits) return LITEVAR_ERR_INVALID_ARG;
+  if (!dev_bits || !on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
   const Step& st = plan->steps[step_k - 1];
   const StepSet& ss = st.sets[set];
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -775,7 +847,7 @@ litevar_status_t litevar_plan_materialize_mask(const litevar_plan_t* plan, int32
 }
 
 litevar_status_t litevar_plan_poll_device_status(const litevar_plan_t* plan) {
-  if (!plan) return LITEVAR_ERR_INVALID_ARG;
+  if (!plan || !on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
   int32_t v = 0;
   LV_CUDA(cudaDeviceSynchronize());
   LV_CUDA(cudaMemcpy(&v, plan->d_status, sizeof(v), cudaMemcpyDeviceToHost));
@@ -799,6 +871,7 @@ litevar_status_t litevar_plan_step_kernel(const litevar_plan_t* plan, int32_t st
   const long long units = (long long)plan->n_heads * (st.share ? batch_pairs : 2 * batch_pairs);
   *kernel = plan->kernel == LITEVAR_KERNEL_SIMT ? LITEVAR_KERNEL_SIMT
             : small_mode(plan, st, units)       ? LITEVAR_KERNEL_SMALL
+            : use_row_kernel(plan, st)          ? LITEVAR_KERNEL_TCGEN05_WS
                                                 : LITEVAR_KERNEL_TCGEN05;
   return LITEVAR_OK;
 }

@@ -277,6 +277,7 @@ extern "C" litevar_status_t litevar_attn_forward_static(
   p.sm_scale = sm_scale > 0.f ? sm_scale : 0.125f;
   p.status = &sp->status;
   p.pairs_per_tile = 0;
+  p.units_per_group = units_per_l2_group(p.L_k, p.n_heads * p.batch_computed);
   p.first_tile_zero = 0;
   p.overlap_launch = 0;  // the plan is written by the two kernels launched just above
   return launch_forward_tcgen05(p, a.n_q_tiles, stream);

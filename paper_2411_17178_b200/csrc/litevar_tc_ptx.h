@@ -181,9 +181,9 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
 // instruction stream is what a product of small MMAs waits for (the tensor pipe takes 50 to 65 cycles per step
 // at N <= 128, a step issued through per-step address arithmetic and predicate set-up costs two to three times
 // that), so the offsets are immediates and nothing but the four MMAs depends on anything.
-template <int kAStep, int kBStep>
-__device__ __forceinline__ void mma_ts_x4(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate_first) {
+template <int kA1, int kA2, int kA3, int kB1, int kB2, int kB3>
+__device__ __forceinline__ void mma_ts_x4_at(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate_first) {
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
       "setp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, 1, 0;\n\t"
@@ -193,9 +193,15 @@ __device__ __forceinline__ void mma_ts_x4(uint32_t d_tmem, uint32_t a_tmem, uint
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a1], b1, %3, q;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a2], b2, %3, q;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a3], b3, %3, q;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate_first), "n"(kAStep), "n"(2 * kAStep),
-        "n"(3 * kAStep), "n"(kBStep), "n"(2 * kBStep), "n"(3 * kBStep)
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate_first), "n"(kA1), "n"(kA2), "n"(kA3),
+        "n"(kB1), "n"(kB2), "n"(kB3)
       : "memory");
+}
+template <int kAStep, int kBStep>
+__device__ __forceinline__ void mma_ts_x4(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate_first) {
+  mma_ts_x4_at<kAStep, 2 * kAStep, 3 * kAStep, kBStep, 2 * kBStep, 3 * kBStep>(d_tmem, a_tmem, b_desc, idesc,
+                                                                               accumulate_first);
 }
 // The same with both operands in shared memory (descriptors).
 template <int kAStep, int kBStep>
@@ -284,6 +290,21 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
+}
+
+// Launch order of the tensor-core kernels.  The (batch row, head) units are taken in groups of
+// p.units_per_group; inside a group the CTAs go query-tile pair by pair (heaviest first, the planner's order), all
+// units of the group side by side.  The K/V of one group is what the CTAs resident at one time read: the host
+// sizes the group so that it fits in half of L2, and every K/V tile then comes from DRAM once per step instead of
+// once per wave of CTAs.
+__device__ __forceinline__ void cta_work(const FwdParams& p, int n_ranks, int& rank, int& unit) {
+  const int n_units = p.n_heads * p.batch_computed;
+  const int g_units = p.units_per_group;
+  const int group = blockIdx.x / (g_units * n_ranks);
+  const int r = blockIdx.x - group * (g_units * n_ranks);
+  const int here = min(g_units, n_units - group * g_units);  // the last group may be smaller
+  rank = r / here;
+  unit = group * g_units + (r - rank * here);
 }
 
 // Walk of the union of two ascending key-tile lists (the two halves of the CTA).

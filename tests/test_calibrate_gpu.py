@@ -1,7 +1,8 @@
 """Window calibration kernel (paper Section 2, steps (1)-(3)) against the oracle, through the C ABI.
 
-The maps are non-negative multiples of 1/1024, so every partial sum is exact in fp64 in any order and the
-integer decision "smallest radius whose window mass reaches R_0 of the part's mass" must agree exactly."""
+Most cases use maps that are non-negative multiples of 1/1024: every partial sum is then exact in fp64 in any
+order and the integer decision "smallest radius whose window mass reaches R_0 of the part's mass" must agree
+exactly.  One case uses real softmax rows, where the kernel's fp32 bins round: see the bound there."""
 import numpy as np
 import pytest
 import torch
@@ -103,3 +104,36 @@ def test_calibration_argument_errors():
         with pytest.raises(binding.LitevarError) as e:
             binding.calibrate_windows(**args)
         assert e.value.status == 1
+
+
+@pytest.mark.parametrize("scales,k,n_maps", [(wl.SCALES_256, 10, 24), (wl.SCALES_512, 9, 6)])
+def test_calibration_on_softmax_rows_within_the_fp32_bin_bound(scales, k, n_maps):
+    """Real post-softmax rows (fp32 softmax of seeded scores with a peak near the co-located keys).  The kernel adds
+    up to 256 rows into lane-private fp32 bins before it flushes them in fp64: a bin takes at most 256 x 8 values
+    of one sign, so its relative rounding error is below 2048 x 2^-24 = 1.3e-4, and so is that of any ratio of sums
+    of bins (numerator and denominator err the same way at most once each: 2.5e-4).  R_w must agree with the
+    oracle's within that bound, and the radius wherever the oracle's R_w at the chosen radius and at the one before
+    stay farther than the bound from R_0."""
+    lib_ready()
+    bound = 2.5e-4
+    n_k, L_k = orc.map_shape(scales, k)
+    g = torch.Generator().manual_seed(100 + k)
+    scores = torch.randn(n_maps, n_k, L_k, generator=g) * 1.5
+    near = torch.from_numpy(orc.mask(scales, k, [-1, -1, -1] + [max(1, s // 5) for s in scales[3:]]))
+    scores = scores + 2.5 * near[None].float()
+    maps32 = torch.softmax(scores, dim=-1)
+    maps = maps32.double().numpy()
+    dev = maps32.cuda()
+    for r0 in (0.6, 0.8, 0.95):
+        rad, ratio = binding.calibrate_windows(scales, k, dev, r0, want_ratio=True)
+        ref = orc.calibrate_radius(scales, k, maps, r0)
+        for j in range(4, k + 1):
+            curve = [orc.window_ratio(scales, k, j, w, maps) for w in range(scales[j - 1])]
+            for w, want in enumerate(curve):
+                assert abs(ratio[j - 1, w] - want) <= bound * max(want, 1e-30), (j, w, ratio[j - 1, w], want)
+            w = int(ref[j - 1])
+            clear = abs(curve[w] - r0) > bound and (w == 0 or abs(curve[w - 1] - r0) > bound)
+            if clear:
+                assert int(rad[j - 1]) == w, (r0, j, rad, ref)
+            else:
+                assert abs(int(rad[j - 1]) - w) <= 1

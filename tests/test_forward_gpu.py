@@ -13,9 +13,11 @@ from tests.gpu_util import assert_close, check_sampled, lib_ready, run_forward, 
 
 pytestmark = pytest.mark.gpu
 
-# AUTO is what callers get: the small-step kernel where a step fits it, the tcgen05 kernel elsewhere
-KERNELS = [binding.KERNEL_SIMT, binding.KERNEL_TCGEN05, binding.KERNEL_AUTO]
-KNAME = {binding.KERNEL_SIMT: "simt", binding.KERNEL_TCGEN05: "tcgen05", binding.KERNEL_AUTO: "auto"}
+# AUTO is what callers get: the small-step kernel where a step fits it, one of the two tcgen05 kernels elsewhere
+KERNELS = [binding.KERNEL_SIMT, binding.KERNEL_TCGEN05, binding.KERNEL_TCGEN05_WS, binding.KERNEL_AUTO]
+KNAME = {binding.KERNEL_SIMT: "simt", binding.KERNEL_TCGEN05: "tcgen05", binding.KERNEL_TCGEN05_WS: "tcgen05-row",
+         binding.KERNEL_AUTO: "auto"}
+TC_KERNELS = (binding.KERNEL_TCGEN05, binding.KERNEL_TCGEN05_WS)
 
 
 TILINGS = [binding.TILING_RASTER, binding.TILING_PATCH]
@@ -89,12 +91,14 @@ def test_config4_final_steps_sampled(tiling):
     total = 0
     for k in (8, 9, 10):
         Q = wl.make_q(w, 0, k, batch_rows=2 * B)
-        got, out = run_forward(plan, k, B, Q, Kc, Vc, binding.KERNEL_TCGEN05)
         smp = stratified_samples(plan, k, 2 * B, w.n_heads, w.scales[k - 1], 20 if tiling == binding.TILING_AUTO else 8, rng)
         total += len(smp)
         ref = orc.attention_sampled(w.scales, k, tab[k - 1], Q, Kc, Vc, smp, share_cfg=True)
-        check_sampled(got, ref, smp, f"config 4 step {k}")
-        assert torch.equal(out[:B].view(torch.int16), out[B:].view(torch.int16))
+        # the default tiling with the kernel AUTO picks and with both tcgen05 kernels; patch tiles with both
+        for kernel in ((binding.KERNEL_AUTO,) if tiling == binding.TILING_AUTO else ()) + TC_KERNELS:
+            got, out = run_forward(plan, k, B, Q, Kc, Vc, kernel)
+            check_sampled(got, ref, smp, f"config 4 step {k} {KNAME[kernel]}")
+            assert torch.equal(out[:B].view(torch.int16), out[B:].view(torch.int16))
     assert tiling != binding.TILING_AUTO or total >= 4096
     plan.close()
 
@@ -114,13 +118,16 @@ def test_config5_sampled(rho, tiling):
         plan = binding.Plan(w.scales, n_heads=w.n_heads, rho=rho, tiling=tiling)
     Kc, Vc = wl.make_kv(w, 0)
     Q = wl.make_q(w, 0, 14)
-    got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, binding.KERNEL_TCGEN05)
-    assert np.isfinite(got).all()
     rng = np.random.default_rng(5)
     smp = stratified_samples(plan, 14, 2, w.n_heads, 128, 128 if tiling == binding.TILING_AUTO else 8, rng)
     assert tiling != binding.TILING_AUTO or len(smp) >= 4096
     ref = orc.attention_sampled(w.scales, 14, tab[13], Q, Kc, Vc, smp)
-    check_sampled(got, ref, smp, f"config 5 rho={rho}")
+    # what AUTO launches for the 2K step (the kernel with a softmax thread per query row), then the other kernel
+    assert plan.step_kernel(14, 1) == binding.KERNEL_TCGEN05_WS
+    for kernel in (binding.KERNEL_AUTO, binding.KERNEL_TCGEN05):
+        got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, kernel)
+        assert np.isfinite(got).all()
+        check_sampled(got, ref, smp, f"config 5 rho={rho} {KNAME[kernel]}")
     plan.close()
 
 
@@ -209,6 +216,31 @@ def test_per_head_window_sets_forward():
     plan.close()
 
 
+@pytest.mark.parametrize("batch_pairs", [1, 64], ids=["B1", "B64"])
+def test_per_head_window_sets_on_the_small_step_kernel(batch_pairs):
+    """Two window sets on a step that AUTO gives to the small-step kernel (64 queries x 155 keys), whose list
+    look-up per head runs on the device.  One batch pair leaves SMs to spare (two warps per row group), 64 batch
+    pairs do not (one warp per row group): both builds of the kernel."""
+    lib_ready()
+    scales = (1, 2, 3, 4, 5, 6, 8)
+    H, k = 4, 7
+    tabs = np.stack([orc.window_table(scales, rho=(1, 8)), orc.window_table(scales, rho=(1, 2))])
+    h2s = [1, 0, 0, 1]
+    w = wl.small_workload(scales, n_heads=H, batch_pairs=batch_pairs, share_cfg=True, index=99)
+    plan = binding.Plan(scales, n_heads=H, radius=tabs, n_sets=2, head_to_set=h2s, share_steps=[1] * len(scales))
+    assert plan.step_kernel(k, batch_pairs) == binding.KERNEL_SMALL
+    Kc, Vc = wl.make_kv(w, 0)
+    Q = wl.make_q(w, 0, k)
+    got, out = run_forward(plan, k, batch_pairs, Q, Kc, Vc)
+    for h in range(H):
+        ref = orc.attention_step(scales, k, tabs[h2s[h]][k - 1], Q[:, h:h + 1], Kc[:, h:h + 1], Vc[:, h:h + 1],
+                                 share_cfg=True)
+        assert_close(got[:, h:h + 1], ref, f"head {h}")
+    assert not np.array_equal(orc.mask(scales, k, tabs[0][k - 1]), orc.mask(scales, k, tabs[1][k - 1]))
+    assert torch.equal(out[:batch_pairs].view(torch.int16), out[batch_pairs:].view(torch.int16))
+    plan.close()
+
+
 def test_forward_argument_errors():
     lib_ready()
     scales = (1, 2, 3, 4)
@@ -256,12 +288,13 @@ def test_band_window_2k_sampled():
     plan = binding.Plan(w.scales, n_heads=w.n_heads, shape=binding.WINDOW_BAND, rho=(1, 7))
     Kc, Vc = wl.make_kv(w, 0)
     Q = wl.make_q(w, 0, 14)
-    got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, binding.KERNEL_TCGEN05)
     rng = np.random.default_rng(6)
     smp = stratified_samples(plan, 14, 2, w.n_heads, 128, 128, rng)
     assert len(smp) >= 4096
     ref = orc.attention_sampled(w.scales, 14, tab[13], Q, Kc, Vc, smp, band=True)
-    check_sampled(got, ref, smp, "band 2K")
+    for kernel in TC_KERNELS:
+        got, _ = run_forward(plan, 14, 1, Q, Kc, Vc, kernel)
+        check_sampled(got, ref, smp, f"band 2K {KNAME[kernel]}")
     plan.close()
 
 
@@ -296,25 +329,37 @@ def test_bench_launch_configuration_sampled(cfg, steps, per_unit):
     plan.close()
 
 
+def _expected_tc(plan, k):
+    """The tcgen05 kernel AUTO picks for a step that is not a small one: the kernel with a softmax thread per
+    query row from eight live key tiles per query tile on."""
+    nq, _, npairs = plan.tile_counts(k)
+    return binding.KERNEL_TCGEN05_WS if -(-npairs // nq) >= 8 else binding.KERNEL_TCGEN05
+
+
 def test_step_kernel_selection():
     """AUTO runs the small-step kernel on steps with one query tile, at most two raster key tiles and little
-    work, whatever the batch; the tcgen05 kernel elsewhere; forcing a kernel or patch tiles overrides it."""
+    work, whatever the batch; a tcgen05 kernel elsewhere (the row kernel on long tile lists); forcing a kernel or
+    patch tiles overrides it."""
     lib_ready()
-    S, T, M = binding.KERNEL_SIMT, binding.KERNEL_TCGEN05, binding.KERNEL_SMALL
+    S, T, R, M = binding.KERNEL_SIMT, binding.KERNEL_TCGEN05, binding.KERNEL_TCGEN05_WS, binding.KERNEL_SMALL
     plan = binding.Plan(wl.SCALES_256, n_heads=2)
-    assert [plan.step_kernel(k, 1) for k in range(1, 11)] == [M] * 7 + [T] * 3     # up to 64 x 155
+    assert [plan.step_kernel(k, 1) for k in range(1, 11)] == [M] * 7 + [T] * 3     # up to 64 x 155; short lists
     assert [plan.step_kernel(k, 64) for k in range(1, 11)] == [M] * 7 + [T] * 3
-    plan.set_kernel(T)
-    assert [plan.step_kernel(k) for k in range(1, 11)] == [T] * 10
-    plan.set_kernel(S)
-    assert [plan.step_kernel(k) for k in range(1, 11)] == [S] * 10
+    for forced in (T, R, S):
+        plan.set_kernel(forced)
+        assert [plan.step_kernel(k) for k in range(1, 11)] == [forced] * 10
     plan.close()
     plan = binding.Plan(wl.SCALES_512, n_heads=2)
-    assert [plan.step_kernel(k, 1) for k in range(1, 11)] == [M] * 6 + [T] * 4     # step 7 has two query tiles
-    assert [plan.step_kernel(k, 64) for k in range(1, 11)] == [M] * 6 + [T] * 4
+    want = [M] * 6 + [_expected_tc(plan, k) for k in range(7, 11)]                  # step 7 has two query tiles
+    assert want[6] == T and want[9] == R                                            # 3 and 13 key tiles per query tile
+    assert [plan.step_kernel(k, 1) for k in range(1, 11)] == want
+    assert [plan.step_kernel(k, 64) for k in range(1, 11)] == want
+    plan.close()
+    plan = binding.Plan(wl.SCALES_2K, n_heads=1)
+    assert plan.step_kernel(14, 1) == R
     plan.close()
     plan = binding.Plan(wl.SCALES_256, n_heads=2, tiling=binding.TILING_PATCH)
-    assert [plan.step_kernel(k) for k in range(1, 11)] == [T] * 10   # patch query tiles at every step
+    assert all(plan.step_kernel(k) in (T, R) for k in range(1, 11))   # patch query tiles at every step: no small steps
     plan.close()
     with pytest.raises(binding.LitevarError):
         binding.Plan((1, 2), n_heads=1).step_kernel(3)
@@ -341,7 +386,7 @@ def test_small_step_kernel_shape_extremes(scales, n_global, share):
     for k in range(1, len(scales) + 1):
         n_k, L_k = orc.map_shape(scales, k)
         small = n_k <= 128 and L_k <= 256 and -(-n_k // 16) * -(-L_k // 64) <= 18
-        assert plan.step_kernel(k, B) == (binding.KERNEL_SMALL if small else binding.KERNEL_TCGEN05), (scales, k)
+        assert plan.step_kernel(k, B) == (binding.KERNEL_SMALL if small else _expected_tc(plan, k)), (scales, k)
         assert small or k < len(scales)     # the step each case is about runs on the small-step kernel
         assert np.array_equal(plan.materialize_mask(k), orc.mask(scales, k, tab[k - 1]))
         Q = wl.make_q(w, 0, k)

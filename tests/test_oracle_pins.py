@@ -137,6 +137,9 @@ def test_live_counts_golden_file():
         assert _closed_form_count(scales, k, list(w[k - 1])) == int(kept)
 
 
+TOTALS_2K = {(1, 8): 34218984, (1, 4): 112575328, (1, 2): 321385764}
+
+
 def test_2k_final_step_counts_closed_form():
     for rho in ((1, 8), (1, 4), (1, 2)):
         w = orc.window_table(S2K, rho=rho)
@@ -158,7 +161,11 @@ def test_2k_final_step_counts_closed_form():
                 lc = min(s_j - 1, orc.centre(c, s_j, s_k) + wj) - max(0, orc.centre(c, s_j, s_k) - wj) + 1
                 per += lr * lc
             assert int(m[i].sum()) == per
-        assert 0 < cf < 16384 * 34240
+        # the whole step, enumerated by the oracle in blocks of query rows, equals the closed form and the totals
+        # worked out by hand for this schedule (6.10 %, 20.07 % and 57.29 % of the 16384 x 34240 map)
+        total = sum(int(orc.mask(S2K, 14, w[13], q_rows=range(q0, min(q0 + 1024, 16384))).sum())
+                    for q0 in range(0, 16384, 1024))
+        assert total == cf == TOTALS_2K[rho]
 
 
 def test_mask_invariants():

@@ -172,3 +172,13 @@ def test_band_window_planner_matches_oracle(scales, rho, tiling):
         assert np.array_equal(plan.materialize_mask(k), ref)
         assert plan.stats(k)["live_entries"] == int(ref.sum())
     plan.close()
+
+
+def test_2k_totals_from_the_planner():
+    """Live entries of the 2K step as the device planner counts them: the totals worked out by hand for this
+    schedule (pinned on the CPU side against the oracle's enumeration and the closed form)."""
+    lib_ready()
+    for rho, want in (((1, 8), 34218984), ((1, 4), 112575328), ((1, 2), 321385764)):
+        plan = binding.Plan(wl.SCALES_2K, n_heads=1, rho=rho)
+        assert plan.stats(14)["live_entries"] == want
+        plan.close()
