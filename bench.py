@@ -500,6 +500,63 @@ def measure_qkv8(device, pk):
     return res
 
 
+def measure_kv8(device, pk):
+    """8-bit K/V cache read by the attention kernel itself (litevar_attn_forward_kv8, paper Section 4) against the
+    bf16 cache, on the two workloads whose steps stream their cache from HBM (3 and 4, raster tiles): microseconds
+    per generation's attention and cache bytes per layer."""
+    from paper_2411_17178_b200 import binding
+    out = []
+    for idx in (3, 4):
+        w = wl.WORKLOADS[idx]
+        n_sets = max(2, min(4, sets_needed(w)[0]))
+        bufs = Buffers(w, n_sets, device)
+        share = [1] * len(w.scales) if w.share_cfg else None
+        plan = binding.Plan(w.scales, n_heads=w.n_heads, rho=w.rho, share_steps=share, tiling=binding.TILING_RASTER)
+        k8 = [binding.quantize_rows(bufs.k[i], want_codes=True) for i in range(n_sets)]
+        v8 = [binding.quantize_rows(bufs.v[i], want_codes=True) for i in range(n_sets)]
+        repeat = max(w.n_layers, n_sets)
+        calls = generation_calls(w, n_sets, repeat)
+
+        def gen_bf16():
+            for k, s_ in calls:
+                plan.forward(k, w.batch_pairs, bufs.q[s_][k], k8[s_][0], v8[s_][0], bufs.out[s_][k])
+
+        def gen_kv8():
+            for k, s_ in calls:
+                plan.forward_kv8(k, w.batch_pairs, bufs.q[s_][k], k8[s_][1], k8[s_][2], k8[s_][3], v8[s_][1], v8[s_][2],
+                                 v8[s_][3], bufs.out[s_][k])
+        res = {}
+        for name, fn in (("bf16_cache_auto_kernels", gen_bf16), ("int8_cache", gen_kv8)):
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                fn()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                fn()
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(5):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            res[name + "_us_per_generation"] = round(e0.elapsed_time(e1) / 5 * 1e3 * w.n_layers / repeat, 1)
+        assert plan.poll() == 0
+        rows = 2 * w.batch_pairs * w.n_heads * wl.cache_len(w.scales, max(w.steps))
+        res.update(config=idx, cache_bytes_per_layer_bf16=rows * 2 * 128, cache_bytes_per_layer_int8=rows * 2 * (64 + 8),
+                   note="int8 path: tcgen05 kernel at every step, raster tiles; bf16 path: the kernels AUTO picks on the dequantised cache")
+        out.append(res)
+        plan.close()
+        del bufs, k8, v8
+        torch.cuda.empty_cache()
+    return out
+
+
 def gpu_arm(args):
     from paper_2411_17178_b200 import build as lvbuild
     rank = int(os.environ.get("RANK", "0"))
@@ -526,7 +583,7 @@ def gpu_arm(args):
         # the window calibration kernel alone (for profiler runs); one GPU
         if rank == 0:
             print(json.dumps({"calibration": measure_calibration(device, pk), "qkv8": measure_qkv8(device, pk),
-                              "peaks": pk}), flush=True)
+                              "kv8_cache": measure_kv8(device, pk), "peaks": pk}), flush=True)
         if barrier:
             barrier()
             torch.distributed.destroy_process_group()
@@ -702,6 +759,7 @@ def gpu_arm(args):
         out["plan_us"] = measure_plan_times()
         out["calibration"] = measure_calibration(device, pk)
         out["qkv8"] = measure_qkv8(device, pk)
+        out["kv8_cache"] = measure_kv8(device, pk)
         out["all_configs_detail"] = detail
     # the short table goes out early in the line and the long per-step records last
     order = ["metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",

@@ -140,6 +140,33 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
                                       void* out, const litevar_strides_t* so, void* stream);
 
 /*
+ * Step-k attention on an 8-bit K/V cache (paper Section 4: Q, K and V in attention quantised to 8 bits, the
+ * "QKV8" rows of its tables).  The cache holds, per row of a head, 64 int8 codes, a scale s and a zero point z
+ * as litevar_quantize_rows produces them; a row enters the attention as code * s + z rounded to bf16.  The kernel
+ * evaluates it as fma(code + 32896, s, z - 32896 s): the second operand is rounded once per row, which moves a
+ * widened value by at most 2^-9 of a quantisation step s before the bf16 rounding (litevar_quantize_rows' own
+ * dequantised rows round product and sum separately, so a few operands differ from them by one bf16 unit and the
+ * result agrees with litevar_attn_forward on the dequantised cache closely, not bit for bit).  The cache takes 72
+ * bytes per row instead of 128 and that is what the kernel reads from HBM.  Q is bf16 (quantise-dequantise it
+ * with litevar_quantize_rows or litevar_quantize_qkv if the step's queries are to be 8-bit too).
+ *
+ *   plan, step_k, batch_pairs, Q, sq, out, so, stream   as for litevar_attn_forward
+ *   Kcodes, Vcodes   device int8 [2B, H, >= L_k, 64]; strides `scodes` in bytes (= elements), each a multiple of 16,
+ *                    token stride >= 64, base pointers 16-byte aligned
+ *   Kscale, Kzero, Vscale, Vzero   device fp32 [2B, H, >= L_k]; strides `srow` in elements, token stride must be 1
+ * Runs the tcgen05 kernel for every step: tensor-map copies bring the codes of a tile into the stage, two warps
+ * widen them in place.  The plan must use raster tiles at this step (LITEVAR_TILING_RASTER, or AUTO at grid
+ * sides below 48): else UNSUPPORTED.
+ * Asynchronous, allocates nothing.  Errors: INVALID_ARG (before any launch), UNSUPPORTED, CUDA.
+ */
+litevar_status_t litevar_attn_forward_kv8(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
+                                          const void* Q, const litevar_strides_t* sq, const int8_t* Kcodes,
+                                          const float* Kscale, const float* Kzero, const int8_t* Vcodes,
+                                          const float* Vscale, const float* Vzero, const litevar_strides_t* scodes,
+                                          const litevar_strides_t* srow, void* out, const litevar_strides_t* so,
+                                          void* stream);
+
+/*
  * Step-k attention without a plan object and without any allocation.  The paper has no counterpart:
  * this is a deployment convenience of this library.
  *

@@ -24,7 +24,8 @@ KERNEL_AUTO, KERNEL_SIMT, KERNEL_TCGEN05, KERNEL_SMALL, KERNEL_TCGEN05_WS = 0, 1
 TILING_AUTO, TILING_RASTER, TILING_PATCH = 0, 1, 2
 
 EXPORTS = (
-    "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_static", "litevar_calibrate_windows",
+    "litevar_attn_plan", "litevar_attn_forward", "litevar_attn_forward_kv8", "litevar_attn_forward_static",
+    "litevar_calibrate_windows",
     "litevar_quantize_rows", "litevar_quantize_qkv",
     "litevar_plan_stats", "litevar_plan_tile_counts",
     "litevar_plan_export_tiles", "litevar_plan_export_bounds", "litevar_plan_materialize_mask",
@@ -74,6 +75,10 @@ def load() -> ctypes.CDLL:
     lib.litevar_attn_forward.restype = ctypes.c_int
     lib.litevar_attn_forward.argtypes = [P, I32, I32, P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides),
                                          P, ctypes.POINTER(_Strides), P, ctypes.POINTER(_Strides), P]
+    lib.litevar_attn_forward_kv8.restype = ctypes.c_int
+    lib.litevar_attn_forward_kv8.argtypes = [P, I32, I32, P, ctypes.POINTER(_Strides), P, P, P, P, P, P,
+                                             ctypes.POINTER(_Strides), ctypes.POINTER(_Strides), P,
+                                             ctypes.POINTER(_Strides), P]
     lib.litevar_attn_forward_static.restype = ctypes.c_int
     lib.litevar_attn_forward_static.argtypes = [ctypes.POINTER(I32), I32, I32, I32, ctypes.c_float,
                                                 ctypes.POINTER(_Window), I32, I32, I32,
@@ -219,6 +224,21 @@ class Plan:
                                             self._strides4_ref[2], out.data_ptr(), self._strides4_ref[3], stream_ptr)
         if st != 0:
             _check(st, "litevar_attn_forward")
+
+    def forward_kv8(self, step_k: int, batch_pairs: int, q, k_codes, k_scale, k_zero, v_codes, v_scale, v_zero, out,
+                    stream=None) -> None:
+        """litevar_attn_forward_kv8 on torch CUDA tensors: q/out bf16 [2B, H, n_k, 64]; codes int8 [2B, H, rows, 64]
+        (K and V with the same strides); scales and zero points fp32 [2B, H, rows] (all four with the same strides)."""
+        assert k_codes.stride() == v_codes.stride() and k_codes.stride(3) == 1
+        assert k_scale.stride() == k_zero.stride() == v_scale.stride() == v_zero.stride() and k_scale.stride(2) == 1
+        sc = _Strides(k_codes.stride(0), k_codes.stride(1), k_codes.stride(2))
+        sr = _Strides(k_scale.stride(0), k_scale.stride(1), 1)
+        stream_ptr = _current_raw_stream(q.device.index) if stream is None else getattr(stream, "cuda_stream", stream)
+        st = self._lib.litevar_attn_forward_kv8(
+            self._h, int(step_k), int(batch_pairs), q.data_ptr(), ctypes.byref(_strides(q)), k_codes.data_ptr(),
+            k_scale.data_ptr(), k_zero.data_ptr(), v_codes.data_ptr(), v_scale.data_ptr(), v_zero.data_ptr(),
+            ctypes.byref(sc), ctypes.byref(sr), out.data_ptr(), ctypes.byref(_strides(out)), stream_ptr)
+        _check(st, "litevar_attn_forward_kv8")
 
     def forward_raw(self, step_k, batch_pairs, q_ptr, q_str, k_ptr, k_str, v_ptr, v_str, o_ptr, o_str,
                     stream_ptr) -> int:

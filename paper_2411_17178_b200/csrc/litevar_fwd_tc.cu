@@ -58,10 +58,25 @@ struct Cfg {
   static constexpr int kThreads = 128 + 256 * NH;
   static constexpr uint32_t kTmemCols = 256 * NH;
   static constexpr int kMinCtas = NH == 2 ? 1 : 2;
+  // 8-bit cache build: threads that widen codes (warps 2 and 3).  A third warp behind the softmax warps (96) was
+  // measured slower: 21 warps are allocated as 24, which caps every thread at 80 registers and spills the softmax.
+  static constexpr int kConvThreads = 64;
+  static constexpr int kSoftmaxEnd = 128 + 256 * NH;  // first thread behind the softmax warps
 };
 
-template <int NH>
-struct SharedStorage {
+// 8-bit cache build: the codes of a tile (128 rows of 64 bytes, as the tensor-map copy delivers them, no swizzle)
+// land in the upper half of the bf16 stage they are widened into; only the rows' scales and zero points need
+// storage of their own (empty in the bf16 build).
+constexpr int kCodeTileBytes = kBlockN * kHeadDim;
+template <bool KV8>
+struct CodeStage {};
+template <>
+struct CodeStage<true> {
+  float sz[2][2][2][kBlockN];  // [tile parity][K, V][scale, shifted zero point][row]
+};
+
+template <int NH, bool KV8>
+struct SharedStorage : CodeStage<KV8> {
   static constexpr int kStages = Cfg<NH>::kStages;
   alignas(1024) uint8_t q[NH][kTileBytes];
   alignas(1024) uint8_t k[kStages][kTileBytes];
@@ -69,6 +84,7 @@ struct SharedStorage {
   alignas(1024) uint8_t ones[kTileBytes];  // bf16 1.0 everywhere: second N block of the PV product's B operand
   alignas(8) uint64_t q_full;
   uint64_t k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
+  uint64_t k_codes[kStages], v_codes[kStages];  // 8-bit build: the codes of a stage have landed
   uint64_t s_full[2], p_full[2][2], o_full[2];  // p_full[h][part]: P of the first / last two chunks of each thread
   unsigned long long xslot[2][2][2][kBlockM];  // [tile parity][half][key half][row]: {tile number + 1, partial row max}
   uint32_t tmem_base;
@@ -83,15 +99,144 @@ constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(k
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) |
                               ((uint32_t)(kOutCols >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
 
+// Byte permute of two words (prmt: selector nibbles 0-3 pick bytes of a, 4-7 bytes of b): e.g. selector 0x7650 puts
+// byte 0 of a under the three upper bytes of b.
+__device__ __forceinline__ uint32_t byte_into(uint32_t a, uint32_t b, uint32_t selector) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(selector));
+  return d;
+}
+
+// One tile of codes, already in registers (thread t of NT holds the 16-code chunks t, t + NT, ... of the 128 x 4
+// chunks of a tile) -> bf16 rows in the 128-byte swizzle the tensor-map copies of the bf16 path produce (16-byte
+// chunk c of row m at position c ^ (m & 7)).  Paper Section 4 (8-bit Q/K/V): a row enters the attention as
+// code * s + z, rounded to bf16.
+// The widening takes one fused multiply-add per pair and no integer conversion (that pipe is the exponential
+// pipe): the codes are biased by 128 (one XOR per four); a byte permute puts each biased code u into the second
+// byte of the bit pattern of 2^15, which is the fp32 number 32768 + u; and fma(32768 + u, s, z') with
+// z' = z - 32896 s, rounded once per row, is code * s + z up to the rounding of z': 2^-9 of a quantisation step s,
+// below the bf16 rounding of the result for every code but 0.
+// Consecutive threads write neighbouring chunks of two rows: no bank conflicts.
+template <int NT>
+__device__ __forceinline__ void widen_code_tile(const uint4 (&q)[(4 * kBlockN + NT - 1) / NT], uint8_t* tile,
+                                                const float* scale, const float* shifted_zero, int t) {
+#pragma unroll
+  for (int it = 0; it < (4 * kBlockN + NT - 1) / NT; ++it) {
+    const int id = t + NT * it;
+    if ((4 * kBlockN) % NT != 0 && id >= 4 * kBlockN) break;
+    const int m = id >> 2, c = id & 3;
+    const float sc = scale[m], zs = shifted_zero[m];
+    const float2 sc2 = make_float2(sc, sc), zs2 = make_float2(zs, zs);
+    const uint32_t w[4] = {q[it].x, q[it].y, q[it].z, q[it].w};
+    uint32_t o[8];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t word = w[e] ^ 0x80808080u;
+      const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(byte_into(word, 0x47000000u, 0x7604u)),
+                                                __uint_as_float(byte_into(word, 0x47000000u, 0x7614u))), sc2, zs2);
+      const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(byte_into(word, 0x47000000u, 0x7624u)),
+                                                __uint_as_float(byte_into(word, 0x47000000u, 0x7634u))), sc2, zs2);
+      o[2 * e] = pack_bf16(x01.x, x01.y);
+      o[2 * e + 1] = pack_bf16(x23.x, x23.y);
+    }
+    uint8_t* row = tile + m * 128;
+    *reinterpret_cast<uint4*>(row + (((2 * c) ^ (m & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+    *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ (m & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+  }
+}
+
+// Barrier of the NT conversion threads that also tells whether any of them gave up a wait, so that all take the
+// same way out.
+template <int NT>
+__device__ __forceinline__ bool converters_sync(bool ok) {
+  uint32_t any_failed;
+  asm volatile(
+      "{\n\t.reg .pred pin, pout;\n\tsetp.eq.u32 pin, %1, 0;\n\t"
+      "bar.red.or.pred pout, 2, %2, pin;\n\tselp.u32 %0, 1, 0, pout;\n\t}"
+      : "=r"(any_failed)
+      : "r"((uint32_t)ok), "n"(NT)
+      : "memory");
+  return any_failed == 0u;
+}
+
+// The conversion warps of the 8-bit build.  The producer lane's tensor-map copies put the codes of a K (V) tile into
+// the upper half of the stage; the conversion threads take them into registers, meet at a barrier (nobody reads the codes any
+// more) and write the widened rows over the whole stage.  The rows' scales and zero points come by plain loads one
+// tile ahead (rows past L_k: 0 and 0; their codes arrive as zeros).
 template <int NH>
-__global__ void __launch_bounds__(Cfg<NH>::kThreads, Cfg<NH>::kMinCtas)
+__device__ __forceinline__ void convert_code_tiles(SharedStorage<NH, true>& sm, const FwdParams& p, const SetDesc& sd,
+                                                   int beg0, int end0, int beg1, int end1, int h, int b,
+                                                   volatile int* abort_flag) {
+  constexpr int kStages = Cfg<NH>::kStages;
+  constexpr int NT = Cfg<NH>::kConvThreads;
+  constexpr int kChunks = (4 * kBlockN + NT - 1) / NT;
+  // warps 2 and 3, then the warp behind the softmax warps
+  const int t = threadIdx.x < 128 ? (int)threadIdx.x - 64 : (int)threadIdx.x - Cfg<NH>::kSoftmaxEnd + 64;
+  const int64_t zoff = (int64_t)b * p.z_sb + (int64_t)h * p.z_sh;
+  float rk[2][2], rv[2][2];  // rows t and t + NT of the tile after the one being converted
+  auto fetch_rows = [&](int kt) {
+    const int row0 = p.key_geom ? p.key_geom[kt].a : kt * kBlockN;  // raster tiles only
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (kBlockN % NT != 0 && t + NT * r >= kBlockN) break;
+      const int row = row0 + t + NT * r;
+      const bool valid = row < p.L_k;
+      const int64_t at = zoff + (valid ? row : 0);
+      rk[r][0] = valid ? __ldg(p.k_scale + at) : 0.f;
+      rk[r][1] = valid ? __ldg(p.k_zero + at) : 0.f;
+      rv[r][0] = valid ? __ldg(p.v_scale + at) : 0.f;
+      rv[r][1] = valid ? __ldg(p.v_zero + at) : 0.f;
+    }
+  };
+  auto shifted = [](float zero, float scale) { return fmaf(-32896.f, scale, zero); };  // z' of widen_code_tile
+  auto take_codes = [&](const uint8_t* stage, uint4 (&q)[kChunks]) {
+#pragma unroll
+    for (int it = 0; it < kChunks; ++it)
+      if ((4 * kBlockN) % NT == 0 || t + NT * it < 4 * kBlockN) q[it] = *reinterpret_cast<const uint4*>(stage + kCodeTileBytes + (t + NT * it) * 16);
+  };
+  UnionWalk row_walk, walk;
+  walk.init(sd.pairs, beg0, end0, beg1, end1);
+  row_walk = walk;
+  bool l0, l1;
+  fetch_rows(row_walk.next(l0, l1));  // the list is not empty
+  for (int i = 0; walk.has(); ++i) {
+    (void)walk.next(l0, l1);
+    const int s = i % kStages, par = i & 1;
+    const uint32_t ph = (uint32_t)((i / kStages) & 1);
+    uint4 q[kChunks];
+    bool ok = mbar_wait(&sm.k_codes[s], ph, abort_flag, p.status);
+    if (ok) take_codes(sm.k[s], q);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (kBlockN % NT != 0 && t + NT * r >= kBlockN) break;
+      sm.sz[par][0][0][t + NT * r] = rk[r][0];
+      sm.sz[par][0][1][t + NT * r] = shifted(rk[r][1], rk[r][0]);
+      sm.sz[par][1][0][t + NT * r] = rv[r][0];
+      sm.sz[par][1][1][t + NT * r] = shifted(rv[r][1], rv[r][0]);
+    }
+    if (!converters_sync<NT>(ok)) break;
+    if (row_walk.has()) fetch_rows(row_walk.next(l0, l1));
+    widen_code_tile<NT>(q, sm.k[s], sm.sz[par][0][0], sm.sz[par][0][1], t);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> the tensor pipe's reads
+    mbar_arrive(&sm.k_full[s]);
+    ok = mbar_wait(&sm.v_codes[s], ph, abort_flag, p.status);
+    if (ok) take_codes(sm.v[s], q);
+    if (!converters_sync<NT>(ok)) break;
+    widen_code_tile<NT>(q, sm.v[s], sm.sz[par][1][0], sm.sz[par][1][1], t);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_arrive(&sm.v_full[s]);
+  }
+}
+
+template <int NH, bool KV8>
+__global__ void __launch_bounds__(Cfg<NH>::kThreads + (KV8 ? Cfg<NH>::kConvThreads - 64 : 0), Cfg<NH>::kMinCtas)
 fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ FwdParams p, int n_q_tiles) {
   constexpr int kStages = Cfg<NH>::kStages;
-  constexpr int kThreads = Cfg<NH>::kThreads;
+  constexpr int kThreads = Cfg<NH>::kThreads + (KV8 ? Cfg<NH>::kConvThreads - 64 : 0);
   constexpr uint32_t kTmemCols = Cfg<NH>::kTmemCols;
   extern __shared__ uint8_t smem_raw[];
   constexpr uint32_t kColO = 128 * NH;
-  SharedStorage<NH>& sm = *reinterpret_cast<SharedStorage<NH>*>(
+  SharedStorage<NH, KV8>& sm = *reinterpret_cast<SharedStorage<NH, KV8>*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // 1-D grid, heaviest query-tile pairs first: all (head, batch row) units of a pair are neighbours
@@ -106,9 +251,11 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sm.k_full[s], 1);
+      mbar_init(&sm.k_full[s], KV8 ? Cfg<NH>::kConvThreads : 1);  // 8-bit cache: every conversion thread arrives
       mbar_init(&sm.k_free[s], 1);
-      mbar_init(&sm.v_full[s], 1);
+      mbar_init(&sm.v_full[s], KV8 ? Cfg<NH>::kConvThreads : 1);
+      mbar_init(&sm.k_codes[s], 1);
+      mbar_init(&sm.v_codes[s], 1);
       mbar_init(&sm.v_free[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
@@ -131,7 +278,7 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
     mbar_expect_tx(&sm.q_full, has1 ? 2 * kTileBytes : kTileBytes);
     load_q_tile(sm.q[0], tm, p, qt0, h, b, &sm.q_full);
     if (has1) load_q_tile(sm.q[NH - 1], tm, p, qt1, h, b, &sm.q_full);
-    if (p.first_tile_zero) {  // key tile 0 (cache rows [0,128), raster) heads every list: no look-up needed
+    if (!KV8 && p.first_tile_zero) {  // key tile 0 (cache rows [0,128), raster) heads every list: no look-up needed
       mbar_expect_tx(&sm.k_full[0], kTileBytes);
       tma_load_4d(sm.k[0], &tm.kr, 0, 0, h, b, &sm.k_full[0]);
       mbar_expect_tx(&sm.v_full[0], kTileBytes);
@@ -170,10 +317,17 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
         if (global_ns() - ts > kWaitLimitNs) break;
     } else if (warp == 0 && lane == 0) {
       // ---------------------------------------------------------------- TMA producer
+      // bf16 cache: a copy fills a stage and completes k_full / v_full.  8-bit cache: a copy brings the 8 KB of codes
+      // of a tile into the upper half of the stage and completes k_codes / v_codes; the conversion warps then write
+      // the stage and complete k_full / v_full.
+      constexpr uint32_t kCopyBytes = KV8 ? kCodeTileBytes : kTileBytes;
+      constexpr uint32_t kCopyAt = KV8 ? kCodeTileBytes : 0;
+      auto k_bar = [&](int s) { return KV8 ? &sm.k_codes[s] : &sm.k_full[s]; };
+      auto v_bar = [&](int s) { return KV8 ? &sm.v_codes[s] : &sm.v_full[s]; };
       UnionWalk pw;
       pw.init(sd.pairs, beg0, end0, beg1, end1);
       int issued = 0;
-      if (p.first_tile_zero) {  // item 0 is already on its way
+      if (!KV8 && p.first_tile_zero) {  // item 0 is already on its way
         bool l0, l1;
         (void)pw.next(l0, l1);
         issued = 1;
@@ -183,17 +337,17 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
         const int kt = pw.next(l0, l1);
         const int s = i % kStages, n = i / kStages;
         if (n > 0 && !mbar_wait(&sm.k_free[s], (uint32_t)((n - 1) & 1), abort_flag, p.status)) break;
-        mbar_expect_tx(&sm.k_full[s], kTileBytes);
-        load_kv_tile(sm.k[s], &tm.kr, tm.k2, p, kt, h, b, &sm.k_full[s]);
+        mbar_expect_tx(k_bar(s), kCopyBytes);
+        load_kv_tile(sm.k[s] + kCopyAt, &tm.kr, tm.k2, p, kt, h, b, k_bar(s));
         if (n > 0 && !mbar_wait(&sm.v_free[s], (uint32_t)((n - 1) & 1), abort_flag, p.status)) {
           // the K copy just issued is still in flight
           const unsigned long long ts = global_ns();
-          while (!mbar_try(&sm.k_full[s], (uint32_t)(n & 1)))
+          while (!mbar_try(k_bar(s), (uint32_t)(n & 1)))
             if (global_ns() - ts > kWaitLimitNs) break;
           break;
         }
-        mbar_expect_tx(&sm.v_full[s], kTileBytes);
-        load_kv_tile(sm.v[s], &tm.vr, tm.v2, p, kt, h, b, &sm.v_full[s]);
+        mbar_expect_tx(v_bar(s), kCopyBytes);
+        load_kv_tile(sm.v[s] + kCopyAt, &tm.vr, tm.v2, p, kt, h, b, v_bar(s));
         issued = i + 1;
       }
       if (*abort_flag) {
@@ -203,10 +357,13 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
           if (global_ns() - ts > kWaitLimitNs) break;
         for (int i = issued > kStages ? issued - kStages : 0; i < issued; ++i) {
           const int s = i % kStages, n = i / kStages;
-          while (!(mbar_try(&sm.k_full[s], (uint32_t)(n & 1)) && mbar_try(&sm.v_full[s], (uint32_t)(n & 1))))
+          while (!(mbar_try(k_bar(s), (uint32_t)(n & 1)) && mbar_try(v_bar(s), (uint32_t)(n & 1))))
             if (global_ns() - ts > 2 * kWaitLimitNs) break;
         }
       }
+    } else if (KV8 && warp >= 2 && end1 > beg0) {
+      // ---------------------------------------------------------------- 8-bit cache: widen the codes of each stage
+      if constexpr (KV8) convert_code_tiles<NH>(sm, p, sd, beg0, end0, beg1, end1, h, b, abort_flag);
     } else if (warp == 1 && lane == 0 && end1 > beg0) {
       // ---------------------------------------------------------------- MMA issuer
       const uint64_t q_desc[2] = {make_desc(smem_u32(sm.q[0])), make_desc(smem_u32(sm.q[NH - 1]))};
@@ -275,6 +432,10 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
         prev_phase = ph;
       }
     }
+  } else if (KV8 && (int)threadIdx.x >= Cfg<NH>::kSoftmaxEnd) {
+    // the conversion warp behind the softmax warps
+    if constexpr (KV8)
+      if (end1 > beg0) convert_code_tiles<NH>(sm, p, sd, beg0, end0, beg1, end1, h, b, abort_flag);
   } else {
     // ------------------------------------------------------------------ softmax + epilogue of one half
     const int hh = (warp - 4) >> 3;        // query half
@@ -520,6 +681,25 @@ bool encode_raster(CUtensorMap* tm, const void* base, int64_t rows, int64_t head
   return r == CUDA_SUCCESS;
 }
 
+// Rank-4 map over a [batch, head, token, 64] tensor of 8-bit codes with byte strides (multiples of 16); box = 128
+// tokens x 64 bytes, rows packed in shared memory without swizzle.  Rows past the last one read as zero.
+bool encode_codes(CUtensorMap* tm, const void* base, int64_t rows, int64_t heads, int64_t batch, int64_t st,
+                  int64_t sh, int64_t sb) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  if (rows < 1) rows = 1;
+  if (heads == 1 && sh < kHeadDim) sh = st * rows;
+  if (batch == 1 && sb < kHeadDim) sb = sh * heads;
+  cuuint64_t gdim[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows, (cuuint64_t)heads, (cuuint64_t)batch};
+  cuuint64_t gstr[3] = {(cuuint64_t)st, (cuuint64_t)sh, (cuuint64_t)sb};
+  cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)kBlockN, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Rank-5 map over the side x side grid of one scale inside a [batch, head, token, 64] tensor: dimensions
 // (64, column, row, head, batch); box = 8 rows x 16 columns x 64, i.e. 128 rows of 128 B in shared memory in
 // row-major patch order.  Cells outside the grid read as zero and are not written.
@@ -540,18 +720,18 @@ bool encode_patch(CUtensorMap* tm, const void* base, int64_t first_token, int64_
   return r == CUDA_SUCCESS;
 }
 
-template <int NH>
+template <int NH, bool KV8>
 litevar_status_t launch_variant(const TensorMaps& tm, const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
-  constexpr int smem_bytes = (int)sizeof(SharedStorage<NH>) + 1024;
+  constexpr int smem_bytes = (int)sizeof(SharedStorage<NH, KV8>) + 1024;
   std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(fwd_tc_kernel<NH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    attr_err = cudaFuncSetAttribute(fwd_tc_kernel<NH, KV8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   });
   if (attr_err != cudaSuccess) return LITEVAR_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((n_q_tiles + NH - 1) / NH) * (unsigned)p.n_heads * (unsigned)p.batch_computed);
-  cfg.blockDim = dim3(Cfg<NH>::kThreads);
+  cfg.blockDim = dim3(Cfg<NH>::kThreads + (KV8 ? Cfg<NH>::kConvThreads - 64 : 0));
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -559,7 +739,7 @@ litevar_status_t launch_variant(const TensorMaps& tm, const FwdParams& p, int n_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = p.overlap_launch ? 1 : 0;  // off when an earlier kernel of the stream writes what the set-up reads
-  if (cudaLaunchKernelEx(&cfg, fwd_tc_kernel<NH>, tm, p, n_q_tiles) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, fwd_tc_kernel<NH, KV8>, tm, p, n_q_tiles) != cudaSuccess) {
     (void)cudaGetLastError();
     return LITEVAR_ERR_CUDA;
   }
@@ -596,7 +776,22 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
   // ... and so does a step whose lists are short (set-up and drain weigh more than the shared K/V staging saves)
   const bool lite = (n_q_tiles == 1 && units > n_sm) ||
                     (units * n_q_tiles >= 2LL * n_sm && p.pairs_per_tile > 0 && p.pairs_per_tile <= 14);
-  return lite ? launch_variant<1>(tm, p, n_q_tiles, stream) : launch_variant<2>(tm, p, n_q_tiles, stream);
+  return lite ? launch_variant<1, false>(tm, p, n_q_tiles, stream) : launch_variant<2, false>(tm, p, n_q_tiles, stream);
+}
+
+litevar_status_t launch_forward_tcgen05_kv8(const FwdParams& p, int n_q_tiles, cudaStream_t stream) {
+  TensorMaps tm;
+  memset(&tm, 0, sizeof(tm));
+  // the raster maps of K and V cover the code tensors here
+  if (!encode_raster(&tm.q, p.q, p.n_k, p.n_heads, p.batch_computed, p.q_st, p.q_sh, p.q_sb) ||
+      !encode_codes(&tm.kr, p.k8, p.L_k, p.n_heads, p.batch_computed, p.c_st, p.c_sh, p.c_sb) ||
+      !encode_codes(&tm.vr, p.v8, p.L_k, p.n_heads, p.batch_computed, p.c_st, p.c_sh, p.c_sb))
+    return LITEVAR_ERR_INVALID_ARG;
+  const int n_sm = current_sm_count();
+  const long long units = (long long)p.n_heads * p.batch_computed;
+  // two query tiles per CTA wherever there are two: a widened K/V tile then serves both
+  const bool lite = n_q_tiles == 1 && units > n_sm;
+  return lite ? launch_variant<1, true>(tm, p, n_q_tiles, stream) : launch_variant<2, true>(tm, p, n_q_tiles, stream);
 }
 
 }  // namespace litevar

@@ -111,6 +111,12 @@ struct FwdParams {
   int32_t* status;              // device word, set non-zero when a bounded wait expires
   int32_t pairs_per_tile;       // average live key tiles per query tile (0: unknown); picks the kernel build
   int32_t first_tile_zero;      // 1: every query tile's list starts with key tile 0 (its copies start at once)
+  // 8-bit K/V cache (litevar_attn_forward_kv8): int8 codes [2B, H, rows, 64] with byte strides c_*, and one fp32
+  // scale and zero point per row, [2B, H, rows] with strides z_sb, z_sh (rows contiguous); k and v are unused
+  const int8_t* k8;
+  const int8_t* v8;
+  const float *k_scale, *k_zero, *v_scale, *v_zero;
+  int64_t c_sb, c_sh, c_st, z_sb, z_sh;
   int32_t units_per_group;      // launch order of the tensor-core kernels: (batch row, head) units per L2 group
   int32_t overlap_launch;       // 1: the tensor-core kernel may start its set-up before the previous kernel of the
                                 // stream has finished (the plan it reads was complete long before)
@@ -165,6 +171,8 @@ cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, in
 
 // Tensor-core path.  Returns LITEVAR_OK or an error status (tensor-map encoding can fail).
 litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
+// The same kernel reading an 8-bit K/V cache (p.k8 ...; raster tiles only).
+litevar_status_t launch_forward_tcgen05_kv8(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
 // The same path with one softmax thread per query row (register reallocation between warpgroups).
 litevar_status_t launch_forward_ws(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
 

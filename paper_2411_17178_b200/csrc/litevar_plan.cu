@@ -676,29 +676,14 @@ litevar_status_t litevar_attn_plan(const int32_t* scales, int32_t n_scales, int3
   return LITEVAR_OK;
 }
 
-litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
-                                      const void* Q, const litevar_strides_t* sq, const void* Kc,
-                                      const litevar_strides_t* sk, const void* Vc, const litevar_strides_t* sv,
-                                      void* out, const litevar_strides_t* so, void* stream_) {
-  if (!plan || !Q || !Kc || !Vc || !out) return LITEVAR_ERR_INVALID_ARG;
-  if (step_k < 1 || step_k > plan->sched.n_scales || batch_pairs < 1) return LITEVAR_ERR_INVALID_ARG;
-  if (!strides_ok(sq) || !strides_ok(sk) || !strides_ok(sv) || !strides_ok(so)) return LITEVAR_ERR_INVALID_ARG;
-  if (((uintptr_t)Q | (uintptr_t)Kc | (uintptr_t)Vc | (uintptr_t)out) & 15) return LITEVAR_ERR_INVALID_ARG;
-  if (!on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
-  const Step& st = plan->steps[step_k - 1];
-  FwdParams p;
+// Launch parameters of a step that do not depend on the tensors.
+static void fill_step_params(const litevar_plan_t* plan, const Step& st, int32_t step_k, int32_t batch_pairs,
+                             FwdParams& p) {
+  memset(&p, 0, sizeof(p));
   p.sets = st.d_sets;
   p.head_to_set = plan->n_sets > 1 ? plan->d_head_to_set : nullptr;
   p.set0 = SetDesc{st.sets[0].d_row_ptr, st.sets[0].d_pairs, st.sets[0].d_mask};
   p.order = st.sets[0].d_order;
-  p.q = static_cast<const uint16_t*>(Q);
-  p.k = static_cast<const uint16_t*>(Kc);
-  p.v = static_cast<const uint16_t*>(Vc);
-  p.out = static_cast<uint16_t*>(out);
-  p.q_sb = sq->batch; p.q_sh = sq->head; p.q_st = sq->token;
-  p.k_sb = sk->batch; p.k_sh = sk->head; p.k_st = sk->token;
-  p.v_sb = sv->batch; p.v_sh = sv->head; p.v_st = sv->token;
-  p.o_sb = so->batch; p.o_sh = so->head; p.o_st = so->token;
   p.n_k = st.n_k;
   p.L_k = st.L_k;
   p.n_heads = plan->n_heads;
@@ -723,6 +708,28 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   for (const StepSet& ss : st.sets) p.first_tile_zero &= ss.first_tile_zero ? 1 : 0;
   p.pairs_per_tile = (st.sets[0].n_pairs + st.n_q_tiles - 1) / st.n_q_tiles;
   p.units_per_group = units_per_l2_group(st.L_k, p.n_heads * p.batch_computed);
+}
+
+litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
+                                      const void* Q, const litevar_strides_t* sq, const void* Kc,
+                                      const litevar_strides_t* sk, const void* Vc, const litevar_strides_t* sv,
+                                      void* out, const litevar_strides_t* so, void* stream_) {
+  if (!plan || !Q || !Kc || !Vc || !out) return LITEVAR_ERR_INVALID_ARG;
+  if (step_k < 1 || step_k > plan->sched.n_scales || batch_pairs < 1) return LITEVAR_ERR_INVALID_ARG;
+  if (!strides_ok(sq) || !strides_ok(sk) || !strides_ok(sv) || !strides_ok(so)) return LITEVAR_ERR_INVALID_ARG;
+  if (((uintptr_t)Q | (uintptr_t)Kc | (uintptr_t)Vc | (uintptr_t)out) & 15) return LITEVAR_ERR_INVALID_ARG;
+  if (!on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
+  const Step& st = plan->steps[step_k - 1];
+  FwdParams p;
+  fill_step_params(plan, st, step_k, batch_pairs, p);
+  p.q = static_cast<const uint16_t*>(Q);
+  p.k = static_cast<const uint16_t*>(Kc);
+  p.v = static_cast<const uint16_t*>(Vc);
+  p.out = static_cast<uint16_t*>(out);
+  p.q_sb = sq->batch; p.q_sh = sq->head; p.q_st = sq->token;
+  p.k_sb = sk->batch; p.k_sh = sk->head; p.k_st = sk->token;
+  p.v_sb = sv->batch; p.v_sh = sv->head; p.v_st = sv->token;
+  p.o_sb = so->batch; p.o_sh = so->head; p.o_st = so->token;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (const int mode = small_mode(plan, st, (long long)p.n_heads * p.batch_computed)) {
     if (launch_forward_small(p, st.sets[0].small, mode, plan->n_sm, stream) != cudaSuccess) {
@@ -741,6 +748,37 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
   }
   if (use_row_kernel(plan, st)) return launch_forward_ws(p, st.n_q_tiles, stream);
   return launch_forward_tcgen05(p, st.n_q_tiles, stream);
+}
+
+litevar_status_t litevar_attn_forward_kv8(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,
+                                          const void* Q, const litevar_strides_t* sq, const int8_t* Kcodes,
+                                          const float* Kscale, const float* Kzero, const int8_t* Vcodes,
+                                          const float* Vscale, const float* Vzero, const litevar_strides_t* scodes,
+                                          const litevar_strides_t* srow, void* out, const litevar_strides_t* so,
+                                          void* stream_) {
+  if (!plan || !Q || !Kcodes || !Kscale || !Kzero || !Vcodes || !Vscale || !Vzero || !out || !scodes || !srow)
+    return LITEVAR_ERR_INVALID_ARG;
+  if (step_k < 1 || step_k > plan->sched.n_scales || batch_pairs < 1) return LITEVAR_ERR_INVALID_ARG;
+  if (!strides_ok(sq) || !strides_ok(so)) return LITEVAR_ERR_INVALID_ARG;
+  if (scodes->batch < 0 || scodes->head < 0 || scodes->token < kHeadDim || (scodes->batch | scodes->head | scodes->token) & 15)
+    return LITEVAR_ERR_INVALID_ARG;  // every code row starts on a 16-byte boundary
+  if (srow->batch < 0 || srow->head < 0 || srow->token != 1) return LITEVAR_ERR_INVALID_ARG;
+  if (((uintptr_t)Q | (uintptr_t)Kcodes | (uintptr_t)Vcodes | (uintptr_t)out) & 15) return LITEVAR_ERR_INVALID_ARG;
+  if (((uintptr_t)Kscale | (uintptr_t)Kzero | (uintptr_t)Vscale | (uintptr_t)Vzero) & 3) return LITEVAR_ERR_INVALID_ARG;
+  if (!on_plan_device(plan)) return LITEVAR_ERR_INVALID_ARG;
+  const Step& st = plan->steps[step_k - 1];
+  if (st.q_patch || st.first_patch != step_k) return LITEVAR_ERR_UNSUPPORTED;  // raster tiles only
+  FwdParams p;
+  fill_step_params(plan, st, step_k, batch_pairs, p);
+  p.q = static_cast<const uint16_t*>(Q);
+  p.out = static_cast<uint16_t*>(out);
+  p.q_sb = sq->batch; p.q_sh = sq->head; p.q_st = sq->token;
+  p.o_sb = so->batch; p.o_sh = so->head; p.o_st = so->token;
+  p.k8 = Kcodes; p.v8 = Vcodes;
+  p.k_scale = Kscale; p.k_zero = Kzero; p.v_scale = Vscale; p.v_zero = Vzero;
+  p.c_sb = scodes->batch; p.c_sh = scodes->head; p.c_st = scodes->token;
+  p.z_sb = srow->batch; p.z_sh = srow->head;
+  return launch_forward_tcgen05_kv8(p, st.n_q_tiles, static_cast<cudaStream_t>(stream_));
 }
 
 static litevar_status_t check_step_set(const litevar_plan_t* plan, int32_t step_k, int32_t set) {

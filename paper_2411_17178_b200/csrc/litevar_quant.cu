@@ -43,20 +43,10 @@ struct QuantArgs {
   float* zero;
 };
 
-// round((x - z) / s) with the IEEE division, for four values (the slow path of the kernel below)
-__device__ __noinline__ float4 exact_codes4(float4 x, float z, float s1) {
-  float4 r;
-  r.x = __fsub_rn(__fadd_rn(__fdiv_rn(__fsub_rn(x.x, z), s1), 12582912.f), 12582912.f);
-  r.y = __fsub_rn(__fadd_rn(__fdiv_rn(__fsub_rn(x.y, z), s1), 12582912.f), 12582912.f);
-  r.z = __fsub_rn(__fadd_rn(__fdiv_rn(__fsub_rn(x.z, z), s1), 12582912.f), 12582912.f);
-  r.w = __fsub_rn(__fadd_rn(__fdiv_rn(__fsub_rn(x.w, z), s1), 12582912.f), 12582912.f);
-  return r;
-}
-
 // kQuantRowsPerGroup rows per 8-thread group: that many 16-byte loads in flight per thread.  Four for large
 // tensors (bandwidth), one for the few rows of a single step (more threads, shorter latency chain).
 template <int kQuantRowsPerGroup>
-__global__ void __launch_bounds__(kQuantThreads) quant_rows_kernel(QuantArgs a) {
+__global__ void __launch_bounds__(kQuantThreads, 4) quant_rows_kernel(QuantArgs a) {
   // the rows were written by earlier work of the stream; a launch with programmatic serialisation starts early
   asm volatile("griddepcontrol.launch_dependents;");
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -116,22 +106,23 @@ __global__ void __launch_bounds__(kQuantThreads) quant_rows_kernel(QuantArgs a) 
     float c[8];
     uint32_t packed[4];
     // round to nearest even without the conversion pipe: adding and subtracting 1.5 * 2^23 is exact rounding
-    // to an integer for |y| < 2^22, and |y| stays near 2^(B-1) here.  |y| <= 2^(B-1) + 1, so two units in the
-    // last place are at most 2^-14: an estimate farther than 2^-12 from a half-integer rounds as the exact
-    // quotient does.  Rows with an estimate closer than that (few) are redone with the IEEE division.
-    bool near_tie = !(s1 > 1e-30f);  // a step so small that its reciprocal is not a normal number: divide
+    // to an integer for |y| < 2^22, and |y| stays near 2^(B-1) here.  The estimate y = (x - z) * (1 / s) is within
+    // |y| * 2^-23 < 2^-15.9 of the true quotient and the correctly rounded quotient within 2^-17 of it, so an
+    // estimate farther than 2^-14 from a half-integer rounds as the IEEE quotient does; a thread with an estimate
+    // closer than that redoes its eight values with the division.  So does every thread of a row whose step is so
+    // small that its reciprocal is not a normal number.
+    bool divide = !(s1 > 1e-30f);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const float y = __fmul_rn(__fsub_rn(v[i], z), r);
       const float n = __fsub_rn(__fadd_rn(y, 12582912.f), 12582912.f);
-      near_tie |= fabsf(__fsub_rn(y, n)) > 0.5f - 0.000244140625f;
+      divide |= fabsf(__fsub_rn(y, n)) > 0.5f - 0.00006103515625f;
       c[i] = n;
     }
-    if (near_tie) {  // rare: kept out of line so that the common path keeps its registers
-      const float4 lo = exact_codes4(make_float4(v[0], v[1], v[2], v[3]), z, s1);
-      const float4 hi = exact_codes4(make_float4(v[4], v[5], v[6], v[7]), z, s1);
-      c[0] = lo.x; c[1] = lo.y; c[2] = lo.z; c[3] = lo.w;
-      c[4] = hi.x; c[5] = hi.y; c[6] = hi.z; c[7] = hi.w;
+    if (divide) {  // rare (one thread-row in a thousand): all eight values again, with the IEEE division
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        c[i] = __fsub_rn(__fadd_rn(__fdiv_rn(__fsub_rn(v[i], z), s1), 12582912.f), 12582912.f);
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) c[i] = s > 0.f ? fminf(fmaxf(c[i], a.lo), a.hi) : 0.f;

@@ -9,7 +9,7 @@ import torch
 
 from oracle import litevar_oracle as orc
 from paper_2411_17178_b200 import binding, workloads as wl
-from tests.gpu_util import assert_close, lib_ready
+from tests.gpu_util import assert_close, errors, lib_ready
 
 pytestmark = pytest.mark.gpu
 
@@ -128,4 +128,93 @@ def test_attention_on_8bit_qkv(k):
     # check above does exercise it
     plain = orc.attention_step(scales, k, tab[k - 1], Q, Kc, Vc)
     assert 0.03 < np.abs(ref - plain).max() < 0.4
+    plan.close()
+
+
+def _cache8(t, rows_extra=0):
+    """Quantise a bf16 cache tensor on the device: (codes, scale, zero, dequantised bf16)."""
+    out, codes, scale, zero = binding.quantize_rows(t, want_codes=True)
+    return codes, scale, zero, out
+
+
+@pytest.mark.parametrize("scales,H,B,share,steps", [
+    (wl.SCALES_256, 3, 1, True, (1, 3, 5, 7, 8, 9, 10)),      # small and large steps, shared
+    (wl.SCALES_512, 2, 1, False, (7, 9, 10)),                 # several query tiles, long lists, unshared
+    ((1, 2, 3, 4, 6, 9, 13, 18, 24), 2, 2, True, (8, 9)),     # ragged last query and key tiles
+], ids=["256px", "512px", "ragged"])
+def test_attention_reads_the_8bit_cache(scales, H, B, share, steps):
+    """litevar_attn_forward_kv8: the attention kernel itself reads int8 codes, scales and zero points and widens
+    them on the way into its shared-memory stages.  Its output must agree closely with the bf16 entry point run
+    on the dequantised cache, and within the parity tolerance with the oracle's attention on the oracle's
+    dequantised tensors.  The cache tensors are longer than L_k and their tail is poisoned."""
+    lib_ready()
+    K = len(scales)
+    L = orc.map_shape(scales, K)[1]
+    Kc = _rows((2 * B, H, L + 40, 64), 700 + K, "offset")
+    Vc = _rows((2 * B, H, L + 40, 64), 800 + K, "normal")
+    kc8, ks, kz, kdq = _cache8(Kc.cuda())
+    vc8, vs, vz, vdq = _cache8(Vc.cuda())
+    plan = binding.Plan(scales, n_heads=H, share_steps=[1] * K if share else None, tiling=binding.TILING_RASTER)
+    tab = orc.window_table(scales)
+    kdq_h = torch.from_numpy(orc.quantize_rows(Kc.float().numpy())[3])
+    vdq_h = torch.from_numpy(orc.quantize_rows(Vc.float().numpy())[3])
+    assert np.array_equal(kdq.float().cpu().numpy(), kdq_h.numpy())
+    for k in steps:
+        n_k, L_k = orc.map_shape(scales, k)
+        Q = _rows((2 * B, H, n_k, 64), 900 + k, "normal")
+        qd = binding.quantize_rows(Q.cuda())                  # 8-bit queries too (Section 4: Q, K and V)
+        # rows beyond L_k must never reach the result: poison them in the 8-bit cache
+        kc8p, ksp = kc8.clone(), ks.clone()
+        kc8p[:, :, L_k:] = 127
+        ksp[:, :, L_k:] = float("nan")
+        want = torch.full(qd.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        plan.set_kernel(binding.KERNEL_TCGEN05)
+        plan.forward(k, B, qd, kdq, vdq, want)
+        got = torch.full(qd.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        plan.forward_kv8(k, B, qd, kc8p, ksp, kz, vc8, vs, vz, got)
+        torch.cuda.synchronize()
+        assert plan.poll() == 0
+        # the widening rounds code * s + z once (a fused multiply-add on a shifted zero point) where the quantiser's
+        # dequantised rows round product and sum separately: a few operands differ by one bf16 unit, so the two
+        # outputs agree far inside the parity tolerance but not bit for bit
+        ma, rl = errors(got.double().cpu().numpy(), want.double().cpu().numpy())
+        assert ma <= 8e-3 and rl <= 3e-3, f"step {k}: 8-bit cache path against the bf16 path: {ma:.2e} {rl:.2e}"
+        qdq_h = torch.from_numpy(orc.quantize_rows(Q.float().numpy())[3])
+        ref = orc.attention_step(scales, k, tab[k - 1], qdq_h, kdq_h, vdq_h, share_cfg=share)
+        assert_close(got.double().cpu().numpy(), ref, f"8-bit cache step {k}")
+        if share:
+            assert torch.equal(got[:B].view(torch.int16), got[B:].view(torch.int16))
+    plan.close()
+
+
+def test_8bit_cache_argument_errors():
+    lib_ready()
+    scales = wl.SCALES_2K
+    plan = binding.Plan(scales, n_heads=1)                    # patch tiles at the last steps
+    q = torch.zeros(2, 1, 16384, 64, dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros(2, 1, 8, 64, dtype=torch.int8, device="cuda")       # never dereferenced
+    z = torch.zeros(2, 1, 8, dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.LitevarError) as e:
+        plan.forward_kv8(14, 1, q, c, z, z, c, z, z, q)
+    assert e.value.status == 2
+    plan.close()
+    plan = binding.Plan((1, 2, 3, 4), n_heads=1)
+    q = torch.zeros(2, 1, 16, 64, dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros(2, 1, 30, 64, dtype=torch.int8, device="cuda")
+    z = torch.zeros(2, 1, 30, dtype=torch.float32, device="cuda")
+    plan.forward_kv8(4, 1, q, c, z, z, c, z, z, q)                       # fine
+    with pytest.raises(binding.LitevarError) as e:
+        plan.forward_kv8(5, 1, q, c, z, z, c, z, z, q)
+    assert e.value.status == 1
+    lib = binding.load()
+    import ctypes
+    sq, sc, sr = binding._strides(q), binding._Strides(1920, 1920, 64), binding._Strides(30, 30, 1)
+    bad = binding._Strides(1920, 1920, 72)                               # rows not on 16-byte boundaries
+    args = lambda codes, srow: (plan._h, 4, 1, q.data_ptr(), ctypes.byref(sq), c.data_ptr(), z.data_ptr(), z.data_ptr(),
+                                c.data_ptr(), z.data_ptr(), z.data_ptr(), ctypes.byref(codes), ctypes.byref(srow),
+                                q.data_ptr(), ctypes.byref(sq), None)
+    assert lib.litevar_attn_forward_kv8(*args(sc, sr)) == 0
+    assert lib.litevar_attn_forward_kv8(*args(bad, sr)) == 1
+    assert lib.litevar_attn_forward_kv8(*args(sc, binding._Strides(30, 30, 2))) == 1
+    torch.cuda.synchronize()
     plan.close()
