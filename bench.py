@@ -2,7 +2,7 @@
 """Benchmark of the LiteVAR attention path (multi-diagonal window mask + CFG sharing) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference] [--no-extras]
-                    [--kernel-only] [--calibration] [--dense] [--rho NUM DEN]
+                    [--kernel-only] [--calibration] [--kv8 [IDX ...]] [--dense] [--rho NUM DEN]
 
 A "step" is one pass of the whole hot path over one batch: one full generation's attention,
 i.e. every scale step of every layer of the chosen workload (for the single-call workloads 1 and
@@ -28,6 +28,8 @@ plan_us          microseconds litevar_attn_plan takes per schedule (device plann
 calibration      the window calibration kernel against the HBM roofline (also: --calibration alone)
 qkv8             the 8-bit Q/K/V row quantiser against the HBM roofline, and the 256px generation
                  with Q and the appended K/V rows quantised before every call
+kv8_cache        the attention reading an 8-bit K/V cache (int8 codes + scale and zero point per row) against the
+                 same steps on the bf16 cache, workloads 3 and 4 (also: --kv8 alone)
 
 With --impl reference the oracle itself is timed (rank 0 only) and printed in the same format.
 """
@@ -79,7 +81,8 @@ KERNEL_NAMES = {1: "fwd_simt_kernel", 2: "fwd_tc_kernel", 3: "fwd_small_kernel",
 
 def recorded_traffic(key):
     """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) recorded in
-    profiles/traffic.txt under `key`, or None when the kernel sources have changed since the counters were taken."""
+    profiles/traffic.txt under `key` (workload.variant.kernel.bytes_per_launch), or None when there is no such
+    record or the kernel sources have changed since the counters were taken."""
     path = os.path.join(ROOT, "profiles", "traffic.txt")
     try:
         kv = dict(l.strip().split("=", 1) for l in open(path) if "=" in l and not l.startswith("#"))
@@ -500,13 +503,13 @@ def measure_qkv8(device, pk):
     return res
 
 
-def measure_kv8(device, pk):
+def measure_kv8(device, pk, configs=(3, 4), reps=5, warm=3):
     """8-bit K/V cache read by the attention kernel itself (litevar_attn_forward_kv8, paper Section 4) against the
     bf16 cache, on the two workloads whose steps stream their cache from HBM (3 and 4, raster tiles): microseconds
     per generation's attention and cache bytes per layer."""
     from paper_2411_17178_b200 import binding
     out = []
-    for idx in (3, 4):
+    for idx in configs:
         w = wl.WORKLOADS[idx]
         n_sets = max(2, min(4, sets_needed(w)[0]))
         bufs = Buffers(w, n_sets, device)
@@ -536,16 +539,16 @@ def measure_kv8(device, pk):
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
                 fn()
-            for _ in range(3):
+            for _ in range(warm):
                 graph.replay()
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            for _ in range(5):
+            for _ in range(reps):
                 graph.replay()
             e1.record()
             torch.cuda.synchronize()
-            res[name + "_us_per_generation"] = round(e0.elapsed_time(e1) / 5 * 1e3 * w.n_layers / repeat, 1)
+            res[name + "_us_per_generation"] = round(e0.elapsed_time(e1) / reps * 1e3 * w.n_layers / repeat, 1)
         assert plan.poll() == 0
         rows = 2 * w.batch_pairs * w.n_heads * wl.cache_len(w.scales, max(w.steps))
         res.update(config=idx, cache_bytes_per_layer_bf16=rows * 2 * 128, cache_bytes_per_layer_int8=rows * 2 * (64 + 8),
@@ -584,6 +587,15 @@ def gpu_arm(args):
         if rank == 0:
             print(json.dumps({"calibration": measure_calibration(device, pk), "qkv8": measure_qkv8(device, pk),
                               "kv8_cache": measure_kv8(device, pk), "peaks": pk}), flush=True)
+        if barrier:
+            barrier()
+            torch.distributed.destroy_process_group()
+        return
+    if args.kv8 is not None:
+        # the 8-bit cache path against the bf16 path alone (for profiler runs); one GPU
+        if rank == 0:
+            print(json.dumps({"kv8_cache": measure_kv8(device, pk, tuple(args.kv8) or (3, 4), args.steps, args.warmup),
+                              "peaks": pk}), flush=True)
         if barrier:
             barrier()
             torch.distributed.destroy_process_group()
@@ -674,7 +686,8 @@ def gpu_arm(args):
         alg = d["bytes"] / d["launches"]
         sec = d["us"] * 1e-6 / d["launches"]
         return {"bound": "hbm", "achieved": round(alg / sec / 1e9, 1), "peak": pk["hbm"], "unit": "GB/s",
-                "frac": round(alg / sec / 1e9 / pk["hbm"], 4), "traffic": recorded_traffic(traffic_key) if traffic_key else None,
+                "frac": round(alg / sec / 1e9 / pk["hbm"], 4),
+                "traffic": recorded_traffic(f"{traffic_key}.{dom}.bytes_per_launch") if traffic_key else None,
                 "kernel": dom, "peak_source": pk["source"], "steps": d["steps"],
                 "launches_per_generation": d["launches"], "share_of_generation_time": round(d["us"] / total_us, 4),
                 "algorithmic_bytes_per_launch": round(alg), "avg_launch_us": round(sec * 1e6, 3),
@@ -693,7 +706,7 @@ def gpu_arm(args):
         useful_l, exec_l = d["useful"] / d["launches"], d["executed"] / d["launches"]
         return {"bound": "tensor", "achieved": round(useful_l / sec / 1e12, 2), "peak": pk["bf16"], "unit": "TFLOP/s",
                 "frac": round(useful_l / sec / 1e12 / pk["bf16"], 4),
-                "traffic": recorded_traffic(traffic_key) if traffic_key else None,
+                "traffic": recorded_traffic(f"{traffic_key}.{dom}.bytes_per_launch") if traffic_key else None,
                 "kernel": dom, "peak_source": pk["source"] + " (burst; a launch is timed alone)",
                 "useful_flop_per_launch": round(useful_l), "executed_flop_per_launch": round(exec_l),
                 "achieved_executed": round(exec_l / sec / 1e12, 2),
@@ -710,7 +723,7 @@ def gpu_arm(args):
 
     timed = kernel_groups(plan, w, bufs, n_sets, repeat, scale, counts)
     default_run = variant == "window" and not args.rho
-    tkey = f"workload{w.index}.{'dense' if variant == 'dense' else 'window'}.bytes_per_launch" if (default_run or variant == "dense") else None
+    tkey = f"workload{w.index}.{'dense' if variant == 'dense' else 'window'}" if (default_run or variant == "dense") else None
     out["roofline"] = tensor_block(timed, tkey) if w.index in (4, 5) else hbm_block(timed, tkey)
 
     if args.kernel_only:
@@ -751,7 +764,7 @@ def gpu_arm(args):
                 rep2 = max(wi.n_layers, n2)
                 out["roofline_hbm_workload2"] = hbm_block(
                     kernel_groups(p2, wi, shared_bufs, n2, rep2, rep2 / wi.n_layers, schedule_counts(p2, wi)),
-                    "workload2.window.bytes_per_launch")
+                    "workload2.window")
                 p2.close()
             del shared_bufs
             torch.cuda.empty_cache()
@@ -893,6 +906,8 @@ def main():
                     help="only the device-timed graph replays (for profiler runs): no eager, end-to-end, "
                          "CPU or all-workload legs")
     ap.add_argument("--calibration", action="store_true", help="only the figures of the window calibration and row quantiser kernels")
+    ap.add_argument("--kv8", type=int, nargs="*", default=None, choices=[3, 4],
+                    help="only the 8-bit K/V cache path against the bf16 path, on the given workloads (default 3 4)")
     ap.add_argument("--rho", type=int, nargs=2, default=None, help="window radius ratio num den (default: the workload's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

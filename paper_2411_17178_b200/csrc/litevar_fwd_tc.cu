@@ -61,7 +61,6 @@ struct Cfg {
   // 8-bit cache build: threads that widen codes (warps 2 and 3).  A third warp behind the softmax warps (96) was
   // measured slower: 21 warps are allocated as 24, which caps every thread at 80 registers and spills the softmax.
   static constexpr int kConvThreads = 64;
-  static constexpr int kSoftmaxEnd = 128 + 256 * NH;  // first thread behind the softmax warps
 };
 
 // 8-bit cache build: the codes of a tile (128 rows of 64 bytes, as the tensor-map copy delivers them, no swizzle)
@@ -170,8 +169,7 @@ __device__ __forceinline__ void convert_code_tiles(SharedStorage<NH, true>& sm, 
   constexpr int kStages = Cfg<NH>::kStages;
   constexpr int NT = Cfg<NH>::kConvThreads;
   constexpr int kChunks = (4 * kBlockN + NT - 1) / NT;
-  // warps 2 and 3, then the warp behind the softmax warps
-  const int t = threadIdx.x < 128 ? (int)threadIdx.x - 64 : (int)threadIdx.x - Cfg<NH>::kSoftmaxEnd + 64;
+  const int t = (int)threadIdx.x - 64;  // warps 2 and 3
   const int64_t zoff = (int64_t)b * p.z_sb + (int64_t)h * p.z_sh;
   float rk[2][2], rv[2][2];  // rows t and t + NT of the tile after the one being converted
   auto fetch_rows = [&](int kt) {
@@ -229,10 +227,10 @@ __device__ __forceinline__ void convert_code_tiles(SharedStorage<NH, true>& sm, 
 }
 
 template <int NH, bool KV8>
-__global__ void __launch_bounds__(Cfg<NH>::kThreads + (KV8 ? Cfg<NH>::kConvThreads - 64 : 0), Cfg<NH>::kMinCtas)
+__global__ void __launch_bounds__(Cfg<NH>::kThreads, Cfg<NH>::kMinCtas)
 fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ FwdParams p, int n_q_tiles) {
   constexpr int kStages = Cfg<NH>::kStages;
-  constexpr int kThreads = Cfg<NH>::kThreads + (KV8 ? Cfg<NH>::kConvThreads - 64 : 0);
+  constexpr int kThreads = Cfg<NH>::kThreads;
   constexpr uint32_t kTmemCols = Cfg<NH>::kTmemCols;
   extern __shared__ uint8_t smem_raw[];
   constexpr uint32_t kColO = 128 * NH;
@@ -432,10 +430,6 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
         prev_phase = ph;
       }
     }
-  } else if (KV8 && (int)threadIdx.x >= Cfg<NH>::kSoftmaxEnd) {
-    // the conversion warp behind the softmax warps
-    if constexpr (KV8)
-      if (end1 > beg0) convert_code_tiles<NH>(sm, p, sd, beg0, end0, beg1, end1, h, b, abort_flag);
   } else {
     // ------------------------------------------------------------------ softmax + epilogue of one half
     const int hh = (warp - 4) >> 3;        // query half
@@ -731,7 +725,7 @@ litevar_status_t launch_variant(const TensorMaps& tm, const FwdParams& p, int n_
   if (attr_err != cudaSuccess) return LITEVAR_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)((n_q_tiles + NH - 1) / NH) * (unsigned)p.n_heads * (unsigned)p.batch_computed);
-  cfg.blockDim = dim3(Cfg<NH>::kThreads + (KV8 ? Cfg<NH>::kConvThreads - 64 : 0));
+  cfg.blockDim = dim3(Cfg<NH>::kThreads);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
