@@ -89,6 +89,13 @@ __device__ __forceinline__ float2 exp2_fma2(float2 x) {
                      __uint_as_float(__float_as_uint(y.y) + (__float_as_uint(t.y) << 23)));
 }
 
+// acc += the two bf16 halves of a packed pair: fp32 additions that take a bf16 operand as it is (no unpacking)
+__device__ __forceinline__ void add_bf16_pair(float2& acc, uint32_t packed) {
+  asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
+      : "+f"(acc.x), "+f"(acc.y)
+      : "r"(packed));
+}
+
 template <int N>
 __device__ __forceinline__ void reg_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
@@ -394,8 +401,8 @@ fwd_ws_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
               // denominator of a row then agree, and a row with one dominant key reproduces that key's V exactly
               const uint32_t ka = pack_bf16(pa.x, pa.y), kb = pack_bf16(pb.x, pb.y);
               if (add_sum) {
-                l2a = __fadd2_rn(l2a, make_float2(__uint_as_float(ka << 16), __uint_as_float(ka & 0xffff0000u)));
-                l2b = __fadd2_rn(l2b, make_float2(__uint_as_float(kb << 16), __uint_as_float(kb & 0xffff0000u)));
+                add_bf16_pair(l2a, ka);
+                add_bf16_pair(l2b, kb);
               }
               pk[(e >> 1) + 0] = ka;
               pk[(e >> 1) + 1] = kb;
