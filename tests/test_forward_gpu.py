@@ -198,6 +198,33 @@ def test_sharp_softmax_and_cache_tail_ignored(kernel):
     plan.close()
 
 
+@pytest.mark.parametrize("kernel", KERNELS, ids=lambda k: KNAME[k])
+def test_dead_keys_with_huge_scores_change_nothing(kernel):
+    """Masking happens before the maximum and the exponentials (Section 2: tokens outside the window are not
+    attended to): keys whose scores dwarf every live score must leave the rows they are dead for untouched.  Two
+    keys of the last scale are scaled by 512; they are live for the queries around them and dead for the rest."""
+    lib_ready()
+    scales = wl.SCALES_256
+    k = 10
+    w = wl.small_workload(scales, n_heads=2, batch_pairs=1, index=92)
+    plan = binding.Plan(scales, n_heads=2, rho=(1, 8))
+    tab = orc.window_table(scales, rho=(1, 8))
+    Kc, Vc = wl.make_kv(w, 0)
+    off = orc.map_shape(scales, k - 1)[1]          # first cache row of the last scale
+    planted = [off + 3 * 16 + 2, off + 12 * 16 + 13]
+    for t in planted:
+        Kc[:, :, t] = (Kc[:, :, t].float() * 512).to(torch.bfloat16)
+    Q = wl.make_q(w, 0, k)
+    got, _ = run_forward(plan, k, 1, Q, Kc, Vc, kernel)
+    ref = orc.attention_step(scales, k, tab[k - 1], Q, Kc, Vc)
+    live = orc.mask(scales, k, tab[k - 1])[:, planted]             # [n_k, 2]
+    untouched = ~live.any(axis=1)
+    assert 100 < untouched.sum() < live.shape[0]
+    assert np.isfinite(got).all()
+    assert_close(got[:, :, untouched], ref[:, :, untouched], "rows for which the planted keys are dead")
+    plan.close()
+
+
 def test_per_head_window_sets_forward():
     lib_ready()
     scales = wl.SCALES_256[:9]
