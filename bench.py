@@ -552,7 +552,7 @@ def measure_kv8(device, pk, configs=(3, 4), reps=5, warm=3):
         assert plan.poll() == 0
         rows = 2 * w.batch_pairs * w.n_heads * wl.cache_len(w.scales, max(w.steps))
         res.update(config=idx, cache_bytes_per_layer_bf16=rows * 2 * 128, cache_bytes_per_layer_int8=rows * 2 * (64 + 8),
-                   note="int8 path: tcgen05 kernel at every step, raster tiles; bf16 path: the kernels AUTO picks on the dequantised cache")
+                   note="int8 path: small-step kernel on the small steps, two-threads-per-row tcgen05 kernel on the others, raster tiles; bf16 path: the kernels AUTO picks on the dequantised cache")
         out.append(res)
         plan.close()
         del bufs, k8, v8

@@ -154,9 +154,10 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
  *   Kcodes, Vcodes   device int8 [2B, H, >= L_k, 64]; strides `scodes` in bytes (= elements), each a multiple of 16,
  *                    token stride >= 64, base pointers 16-byte aligned
  *   Kscale, Kzero, Vscale, Vzero   device fp32 [2B, H, >= L_k]; strides `srow` in elements, token stride must be 1
- * Runs the tcgen05 kernel for every step: tensor-map copies bring the codes of a tile into the stage, two warps
- * widen them in place.  The plan must use raster tiles at this step (LITEVAR_TILING_RASTER, or AUTO at grid
- * sides below 48): else UNSUPPORTED.
+ * Small steps run the small-step kernel, which widens the prefix while it stages it; the others run the
+ * two-threads-per-row tcgen05 kernel: tensor-map copies bring the codes of a tile into the stage, two warps widen
+ * them in place.  The plan must use raster tiles at this step (LITEVAR_TILING_RASTER, or AUTO at grid sides below
+ * 48): else UNSUPPORTED.
  * Asynchronous, allocates nothing.  Errors: INVALID_ARG (before any launch), UNSUPPORTED, CUDA.
  */
 litevar_status_t litevar_attn_forward_kv8(const litevar_plan_t* plan, int32_t step_k, int32_t batch_pairs,

@@ -69,7 +69,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // SPLIT = 1: one warp per 16 query rows.  SPLIT = 2: two warps per 16 query rows, each taking every other
 // 64-key round, merged through shared memory at the end; for launches that leave SMs to spare, where the
 // chain of rounds of a single warp is what the call waits for.
-template <int SPLIT>
+template <int SPLIT, bool KV8>
 __global__ void __launch_bounds__(kSmallMaxWarps * 32 * SPLIT) fwd_small_kernel(FwdParams p, SmallLists lists) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -138,7 +138,33 @@ __global__ void __launch_bounds__(kSmallMaxWarps * 32 * SPLIT) fwd_small_kernel(
   // ---- stage Q and the K/V prefix (written by earlier work of the stream: wait for it first).  blockDim is a
   // multiple of 32, so a thread keeps its 16-byte column (tid % 8) and walks rows.
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  {
+  if constexpr (KV8) {
+    // 8-bit K/V cache (paper Section 4): Q by asynchronous copies as below; the prefix arrives as int8 codes with a
+    // scale and a zero point per row and is widened on the way into the same bf16 rows (16 codes per thread and
+    // chunk: consecutive threads read consecutive 16 bytes of a row).
+    const int row_step = (int)(blockDim.x >> 3);
+    uint16_t* qdst = Qs + (tid & 7) * 8;
+    for (int row = tid >> 3; row < n_k; row += row_step) cp_async16(qdst + row * kRowPad, qsrc + row * q_st);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    const int8_t* kc = p.k8 + b * p.c_sb + h * p.c_sh;
+    const int8_t* vc = p.v8 + b * p.c_sb + h * p.c_sh;
+    const int64_t zoff = b * p.z_sb + h * p.z_sh;
+    for (int c = tid; c < 4 * L_k; c += (int)blockDim.x) {
+      const int row = c >> 2, part = c & 3;
+      const uint4 kq = __ldg(reinterpret_cast<const uint4*>(kc + (int64_t)row * p.c_st) + part);
+      const uint4 vq = __ldg(reinterpret_cast<const uint4*>(vc + (int64_t)row * p.c_st) + part);
+      const float ks = __ldg(p.k_scale + zoff + row), kz = __ldg(p.k_zero + zoff + row);
+      const float vs = __ldg(p.v_scale + zoff + row), vz = __ldg(p.v_zero + zoff + row);
+      uint4 lo, hi;
+      widen_codes16(kq, ks, shifted_zero_point(kz, ks), lo, hi);
+      *reinterpret_cast<uint4*>(Ks + row * kRowPad + part * 16) = lo;
+      *reinterpret_cast<uint4*>(Ks + row * kRowPad + part * 16 + 8) = hi;
+      widen_codes16(vq, vs, shifted_zero_point(vz, vs), lo, hi);
+      *reinterpret_cast<uint4*>(Vs + row * kRowPad + part * 16) = lo;
+      *reinterpret_cast<uint4*>(Vs + row * kRowPad + part * 16 + 8) = hi;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else {
     const int row_step = (int)(blockDim.x >> 3);
     uint16_t* kdst = Ks + (tid & 7) * 8;
     uint16_t* vdst = Vs + (tid & 7) * 8;
@@ -359,14 +385,14 @@ int small_step_mode(int n_k, int L_k, long long units, int n_sm) {
   return units <= n_sm && rounds >= 2 ? 2 : 1;
 }
 
-template <int SPLIT>
+template <int SPLIT, bool KV8>
 static cudaError_t launch_small_variant(const FwdParams& p, const SmallLists& lists, int n_sm, cudaStream_t stream) {
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
   constexpr int kMaxSmem = (kBlockM + 2 * 2 * kBlockN) * kRowPad * 2 + kBlockM * 32 +
                            (SPLIT == 2 ? (kBlockM / 16) * kMergeFloats * 4 : 0);
   std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(fwd_small_kernel<SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    attr_err = cudaFuncSetAttribute(fwd_small_kernel<SPLIT, KV8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
   });
   if (attr_err != cudaSuccess) return attr_err;
   const int q_rows = (p.n_k + 15) / 16 * 16, l_pad = (p.L_k + 15) & ~15;
@@ -387,11 +413,18 @@ static cudaError_t launch_small_variant(const FwdParams& p, const SmallLists& li
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = p.overlap_launch ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, fwd_small_kernel<SPLIT>, p, lists);
+  return cudaLaunchKernelEx(&cfg, fwd_small_kernel<SPLIT, KV8>, p, lists);
 }
 
 cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, int mode, int n_sm, cudaStream_t stream) {
-  return mode == 2 ? launch_small_variant<2>(p, lists, n_sm, stream) : launch_small_variant<1>(p, lists, n_sm, stream);
+  return mode == 2 ? launch_small_variant<2, false>(p, lists, n_sm, stream)
+                   : launch_small_variant<1, false>(p, lists, n_sm, stream);
+}
+
+cudaError_t launch_forward_small_kv8(const FwdParams& p, const SmallLists& lists, int mode, int n_sm,
+                                     cudaStream_t stream) {
+  return mode == 2 ? launch_small_variant<2, true>(p, lists, n_sm, stream)
+                   : launch_small_variant<1, true>(p, lists, n_sm, stream);
 }
 
 }  // namespace litevar

@@ -98,23 +98,11 @@ constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(k
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) |
                               ((uint32_t)(kOutCols >> 3) << 17) | ((uint32_t)(kBlockM >> 4) << 24);
 
-// Byte permute of two words (prmt: selector nibbles 0-3 pick bytes of a, 4-7 bytes of b): e.g. selector 0x7650 puts
-// byte 0 of a under the three upper bytes of b.
-__device__ __forceinline__ uint32_t byte_into(uint32_t a, uint32_t b, uint32_t selector) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(selector));
-  return d;
-}
-
 // One tile of codes, already in registers (thread t of NT holds the 16-code chunks t, t + NT, ... of the 128 x 4
 // chunks of a tile) -> bf16 rows in the 128-byte swizzle the tensor-map copies of the bf16 path produce (16-byte
 // chunk c of row m at position c ^ (m & 7)).  Paper Section 4 (8-bit Q/K/V): a row enters the attention as
 // code * s + z, rounded to bf16.
-// The widening takes one fused multiply-add per pair and no integer conversion (that pipe is the exponential
-// pipe): the codes are biased by 128 (one XOR per four); a byte permute puts each biased code u into the second
-// byte of the bit pattern of 2^15, which is the fp32 number 32768 + u; and fma(32768 + u, s, z') with
-// z' = z - 32896 s, rounded once per row, is code * s + z up to the rounding of z': 2^-9 of a quantisation step s,
-// below the bf16 rounding of the result for every code but 0.
+// The arithmetic is widen_codes16's (one fused multiply-add per pair on a shifted zero point).
 // Consecutive threads write neighbouring chunks of two rows: no bank conflicts.
 template <int NT>
 __device__ __forceinline__ void widen_code_tile(const uint4 (&q)[(4 * kBlockN + NT - 1) / NT], uint8_t* tile,
@@ -124,23 +112,11 @@ __device__ __forceinline__ void widen_code_tile(const uint4 (&q)[(4 * kBlockN + 
     const int id = t + NT * it;
     if ((4 * kBlockN) % NT != 0 && id >= 4 * kBlockN) break;
     const int m = id >> 2, c = id & 3;
-    const float sc = scale[m], zs = shifted_zero[m];
-    const float2 sc2 = make_float2(sc, sc), zs2 = make_float2(zs, zs);
-    const uint32_t w[4] = {q[it].x, q[it].y, q[it].z, q[it].w};
-    uint32_t o[8];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const uint32_t word = w[e] ^ 0x80808080u;
-      const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(byte_into(word, 0x47000000u, 0x7604u)),
-                                                __uint_as_float(byte_into(word, 0x47000000u, 0x7614u))), sc2, zs2);
-      const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(byte_into(word, 0x47000000u, 0x7624u)),
-                                                __uint_as_float(byte_into(word, 0x47000000u, 0x7634u))), sc2, zs2);
-      o[2 * e] = pack_bf16(x01.x, x01.y);
-      o[2 * e + 1] = pack_bf16(x23.x, x23.y);
-    }
+    uint4 lo, hi;
+    widen_codes16(q[it], scale[m], shifted_zero[m], lo, hi);
     uint8_t* row = tile + m * 128;
-    *reinterpret_cast<uint4*>(row + (((2 * c) ^ (m & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-    *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ (m & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+    *reinterpret_cast<uint4*>(row + (((2 * c) ^ (m & 7)) << 4)) = lo;
+    *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ (m & 7)) << 4)) = hi;
   }
 }
 
@@ -186,7 +162,6 @@ __device__ __forceinline__ void convert_code_tiles(SharedStorage<NH, true>& sm, 
       rv[r][1] = valid ? __ldg(p.v_zero + at) : 0.f;
     }
   };
-  auto shifted = [](float zero, float scale) { return fmaf(-32896.f, scale, zero); };  // z' of widen_code_tile
   auto take_codes = [&](const uint8_t* stage, uint4 (&q)[kChunks]) {
 #pragma unroll
     for (int it = 0; it < kChunks; ++it)
@@ -208,9 +183,9 @@ __device__ __forceinline__ void convert_code_tiles(SharedStorage<NH, true>& sm, 
     for (int r = 0; r < 2; ++r) {
       if (kBlockN % NT != 0 && t + NT * r >= kBlockN) break;
       sm.sz[par][0][0][t + NT * r] = rk[r][0];
-      sm.sz[par][0][1][t + NT * r] = shifted(rk[r][1], rk[r][0]);
+      sm.sz[par][0][1][t + NT * r] = shifted_zero_point(rk[r][1], rk[r][0]);
       sm.sz[par][1][0][t + NT * r] = rv[r][0];
-      sm.sz[par][1][1][t + NT * r] = shifted(rv[r][1], rv[r][0]);
+      sm.sz[par][1][1][t + NT * r] = shifted_zero_point(rv[r][1], rv[r][0]);
     }
     if (!converters_sync<NT>(ok)) break;
     if (row_walk.has()) fetch_rows(row_walk.next(l0, l1));

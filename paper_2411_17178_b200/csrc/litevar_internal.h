@@ -168,6 +168,9 @@ cudaError_t launch_forward_simt(const FwdParams& p, int n_q_tiles, cudaStream_t 
 bool small_step_candidate(int n_q_tiles, int n_key_tiles, bool raster_only);
 int small_step_mode(int n_k, int L_k, long long units, int n_sm);
 cudaError_t launch_forward_small(const FwdParams& p, const SmallLists& lists, int mode, int n_sm, cudaStream_t stream);
+// The same kernel reading an 8-bit K/V cache (p.k8 ...).
+cudaError_t launch_forward_small_kv8(const FwdParams& p, const SmallLists& lists, int mode, int n_sm,
+                                     cudaStream_t stream);
 
 // Tensor-core path.  Returns LITEVAR_OK or an error status (tensor-map encoding can fail).
 litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
@@ -175,6 +178,36 @@ litevar_status_t launch_forward_tcgen05(const FwdParams& p, int n_q_tiles, cudaS
 litevar_status_t launch_forward_tcgen05_kv8(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
 // The same path with one softmax thread per query row (register reallocation between warpgroups).
 litevar_status_t launch_forward_ws(const FwdParams& p, int n_q_tiles, cudaStream_t stream);
+
+#ifdef __CUDACC__
+// 8-bit cache rows (paper Section 4): 16 int8 codes of one row -> 16 bf16 values code * s + z, as two 16-byte chunks.
+// One fused multiply-add per pair and no integer conversion (that pipe is the exponential pipe): the codes are biased
+// by 128 (one XOR per four); a byte permute puts each biased code u into the second byte of the bit pattern of 2^15,
+// which is the fp32 number 32768 + u; and fma(32768 + u, s, z') with z' = z - 32896 s (shifted_zero, rounded once
+// per row) is code * s + z up to the rounding of z': 2^-9 of a quantisation step s.
+__device__ __forceinline__ float shifted_zero_point(float zero, float scale) { return fmaf(-32896.f, scale, zero); }
+__device__ __forceinline__ void widen_codes16(const uint4& codes, float scale, float shifted_zero, uint4& lo, uint4& hi) {
+  const float2 sc2 = make_float2(scale, scale), zs2 = make_float2(shifted_zero, shifted_zero);
+  const uint32_t w[4] = {codes.x, codes.y, codes.z, codes.w};
+  uint32_t o[8];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const uint32_t word = w[e] ^ 0x80808080u;
+    uint32_t f[4];
+    // prmt: selector nibbles 0-3 pick bytes of the first operand, 4-7 of the second
+    asm("prmt.b32 %0, %1, %2, 0x7604;" : "=r"(f[0]) : "r"(word), "r"(0x47000000u));
+    asm("prmt.b32 %0, %1, %2, 0x7614;" : "=r"(f[1]) : "r"(word), "r"(0x47000000u));
+    asm("prmt.b32 %0, %1, %2, 0x7624;" : "=r"(f[2]) : "r"(word), "r"(0x47000000u));
+    asm("prmt.b32 %0, %1, %2, 0x7634;" : "=r"(f[3]) : "r"(word), "r"(0x47000000u));
+    const float2 x01 = __ffma2_rn(make_float2(__uint_as_float(f[0]), __uint_as_float(f[1])), sc2, zs2);
+    const float2 x23 = __ffma2_rn(make_float2(__uint_as_float(f[2]), __uint_as_float(f[3])), sc2, zs2);
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[2 * e]) : "f"(x01.y), "f"(x01.x));
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[2 * e + 1]) : "f"(x23.y), "f"(x23.x));
+  }
+  lo = make_uint4(o[0], o[1], o[2], o[3]);
+  hi = make_uint4(o[4], o[5], o[6], o[7]);
+}
+#endif
 
 }  // namespace litevar
 

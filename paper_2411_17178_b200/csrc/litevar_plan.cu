@@ -778,7 +778,15 @@ litevar_status_t litevar_attn_forward_kv8(const litevar_plan_t* plan, int32_t st
   p.k_scale = Kscale; p.k_zero = Kzero; p.v_scale = Vscale; p.v_zero = Vzero;
   p.c_sb = scodes->batch; p.c_sh = scodes->head; p.c_st = scodes->token;
   p.z_sb = srow->batch; p.z_sh = srow->head;
-  return launch_forward_tcgen05_kv8(p, st.n_q_tiles, static_cast<cudaStream_t>(stream_));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (const int mode = small_mode(plan, st, (long long)p.n_heads * p.batch_computed)) {
+    if (launch_forward_small_kv8(p, st.sets[0].small, mode, plan->n_sm, stream) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return LITEVAR_ERR_CUDA;
+    }
+    return LITEVAR_OK;
+  }
+  return launch_forward_tcgen05_kv8(p, st.n_q_tiles, stream);
 }
 
 static litevar_status_t check_step_set(const litevar_plan_t* plan, int32_t step_k, int32_t set) {

@@ -182,6 +182,15 @@ def test_attention_reads_the_8bit_cache(scales, H, B, share, steps):
         qdq_h = torch.from_numpy(orc.quantize_rows(Q.float().numpy())[3])
         ref = orc.attention_step(scales, k, tab[k - 1], qdq_h, kdq_h, vdq_h, share_cfg=share)
         assert_close(got.double().cpu().numpy(), ref, f"8-bit cache step {k}")
+        # under AUTO the small steps read the 8-bit cache in the small-step kernel
+        plan.set_kernel(binding.KERNEL_AUTO)
+        got_auto = torch.full(qd.shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        plan.forward_kv8(k, B, qd, kc8p, ksp, kz, vc8, vs, vz, got_auto)
+        torch.cuda.synchronize()
+        assert plan.poll() == 0
+        assert_close(got_auto.double().cpu().numpy(), ref, f"8-bit cache step {k}, kernel chosen by the plan")
+        small = plan.step_kernel(k, B) == binding.KERNEL_SMALL
+        assert small or torch.equal(got_auto.view(torch.int16), got.view(torch.int16))
         if share:
             assert torch.equal(got[:B].view(torch.int16), got[B:].view(torch.int16))
     plan.close()
