@@ -58,9 +58,10 @@ struct Cfg {
   static constexpr int kThreads = 128 + 256 * NH;
   static constexpr uint32_t kTmemCols = 256 * NH;
   static constexpr int kMinCtas = NH == 2 ? 1 : 2;
-  // 8-bit cache build: threads that widen codes (warps 2 and 3).  A third warp behind the softmax warps (96) was
-  // measured slower: 21 warps are allocated as 24, which caps every thread at 80 registers and spills the softmax.
-  static constexpr int kConvThreads = 64;
+  // 8-bit cache build: threads that widen codes: warps 0, 2 and 3, so that three of the four schedulers share the
+  // work (the copy-issuing lane then sits in warp 1 beside the MMA lane).  A warp behind the softmax warps instead
+  // was measured slower: 21 warps are allocated as 24, which caps every thread at 80 registers and spills the softmax.
+  static constexpr int kConvThreads = 96;
 };
 
 // 8-bit cache build: the codes of a tile (128 rows of 64 bytes, as the tensor-map copy delivers them, no swizzle)
@@ -145,7 +146,10 @@ __device__ __forceinline__ void convert_code_tiles(SharedStorage<NH, true>& sm, 
   constexpr int kStages = Cfg<NH>::kStages;
   constexpr int NT = Cfg<NH>::kConvThreads;
   constexpr int kChunks = (4 * kBlockN + NT - 1) / NT;
-  const int t = (int)threadIdx.x - 64;  // warps 2 and 3
+  const int t = threadIdx.x < 32 ? (int)threadIdx.x : (int)threadIdx.x - 32;  // warp 0, then warps 2 and 3
+  // the scales and zero points may come from the kernel just before this one in the stream: every thread that reads
+  // them waits for it
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int64_t zoff = (int64_t)b * p.z_sb + (int64_t)h * p.z_sh;
   float rk[2][2], rv[2][2];  // rows t and t + NT of the tile after the one being converted
   auto fetch_rows = [&](int kt) {
@@ -288,8 +292,8 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
       const unsigned long long ts = global_ns();
       while (!mbar_try(&sm.q_full, 0u))
         if (global_ns() - ts > kWaitLimitNs) break;
-    } else if (warp == 0 && lane == 0) {
-      // ---------------------------------------------------------------- TMA producer
+    } else if (KV8 ? (warp == 1 && lane == 1) : (warp == 0 && lane == 0)) {
+      // ---------------------------------------------------------------- TMA producer (8-bit build: in the MMA warp)
       // bf16 cache: a copy fills a stage and completes k_full / v_full.  8-bit cache: a copy brings the 8 KB of codes
       // of a tile into the upper half of the stage and completes k_codes / v_codes; the conversion warps then write
       // the stage and complete k_full / v_full.
@@ -334,7 +338,7 @@ fwd_tc_kernel(const __grid_constant__ TensorMaps tm, const __grid_constant__ Fwd
             if (global_ns() - ts > 2 * kWaitLimitNs) break;
         }
       }
-    } else if (KV8 && warp >= 2 && end1 > beg0) {
+    } else if (KV8 && warp != 1 && end1 > beg0) {
       // ---------------------------------------------------------------- 8-bit cache: widen the codes of each stage
       if constexpr (KV8) convert_code_tiles<NH>(sm, p, sd, beg0, end0, beg1, end1, h, b, abort_flag);
     } else if (warp == 1 && lane == 0 && end1 > beg0) {
