@@ -155,7 +155,7 @@ litevar_status_t litevar_attn_forward(const litevar_plan_t* plan, int32_t step_k
  *                    token stride >= 64, base pointers 16-byte aligned
  *   Kscale, Kzero, Vscale, Vzero   device fp32 [2B, H, >= L_k]; strides `srow` in elements, token stride must be 1
  * Small steps run the small-step kernel, which widens the prefix while it stages it; the others run the
- * two-threads-per-row tcgen05 kernel: tensor-map copies bring the codes of a tile into the stage, two warps widen
+ * two-threads-per-row tcgen05 kernel: tensor-map copies bring the codes of a tile into the stage, three warps widen
  * them in place.  The plan must use raster tiles at this step (LITEVAR_TILING_RASTER, or AUTO at grid sides below
  * 48): else UNSUPPORTED.
  * Asynchronous, allocates nothing.  Errors: INVALID_ARG (before any launch), UNSUPPORTED, CUDA.
