@@ -59,9 +59,10 @@ struct Cfg {
   static constexpr uint32_t kTmemCols = 256 * NH;
   static constexpr int kMinCtas = NH == 2 ? 1 : 2;
   // 8-bit cache build: threads that widen codes: warps 0, 2 and 3, so that three of the four schedulers share the
-  // work (the copy-issuing lane then sits in warp 1 beside the MMA lane; inside warp 0 its waits stalled the 31 lanes
-  // beside it, and conversion in the spare lanes of warp 1 delayed the MMA lane: both measured slower).  A warp behind the softmax warps instead
-  // was measured slower: 21 warps are allocated as 24, which caps every thread at 80 registers and spills the softmax.
+  // work; the copy-issuing lane then sits in warp 1 beside the MMA lane.  Measured slower: the issuer inside warp 0
+  // (its waits stall the 31 lanes beside it), conversion in the spare lanes of warp 1 (it delays the MMA lane), and
+  // a conversion warp behind the softmax warps (21 warps are allocated as 24, which caps every thread at 80
+  // registers and spills the softmax).
   static constexpr int kConvThreads = 96;
 };
 
